@@ -1,0 +1,180 @@
+/*
+ * rd.h -- C ABI of the recurrent-depth sampler library for NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the paper's statement of the problem:
+ *   model       e = P(x), s_0 ~ N(0, sigma^2 I), s_i = R(e, s_{i-1}), p = C(s_r)   (Section 3.1)
+ *   KV sharing  one K/V entry per (layer, position), overwritten by the latest pass (Section 3.2)
+ *   prefill     all prompt positions iterate the recurrence together             (Section 3.3)
+ *   AR step     the sequential recurrence, one token per call                    (Section 3.1)
+ *   DF step     one step of the diffusion-forcing sampler: Algorithm 1 (fixed exit) and
+ *               Algorithm 2 with the exit rule of Eq. 3 (adaptive exit), wavefront limiter of
+ *               Section 3.5
+ *
+ * Conventions
+ *   - Every call returns RD_OK (0) or a negative RD_E_* code; nothing throws or aborts across
+ *     this boundary; out-parameters are written only on success.
+ *   - The library owns all device memory it allocates.  The caller owns every buffer it passes;
+ *     buffers are borrowed for the duration of the call only (prompts and weights are copied).
+ *   - "host pointer" / "device pointer" is stated per argument.  Weight pointers may be either
+ *     (copied with cudaMemcpyDefault).
+ *   - Steps are enqueued asynchronously on the session's stream; the calls that read results
+ *     (rd_committed, rd_get_tokens, rd_debug_read, rd_stats) synchronise that stream first.
+ *   - A session is used by one host thread at a time.  One session lives on one GPU: the device
+ *     current when rd_load / rd_session_create are called.
+ *   - All matrices are [out_features, in_features], row-major.
+ */
+#ifndef RD_H_
+#define RD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { RD_F32 = 0, RD_BF16 = 1 };
+
+enum {
+    RD_OK = 0,
+    RD_E_INVALID_ARG = -1, /* null pointer, shape the kernels do not support, bad index      */
+    RD_E_STATE = -2,       /* call out of order (step before prefill, AR inside an open wave) */
+    RD_E_CAPACITY = -3,    /* prompt + budget exceed max_context, window exceeds max_window   */
+    RD_E_OOM = -4,         /* device allocation failed                                        */
+    RD_E_CUDA = -5,        /* a CUDA call or kernel launch failed; see rd_last_cuda_error     */
+    RD_E_TIMEOUT = -6      /* a bounded device-side wait ran out (pipeline barrier)           */
+};
+
+typedef struct rd_model rd_model;     /* opaque: device weights                          */
+typedef struct rd_session rd_session; /* opaque: KV caches, latents, tokens, wavefront   */
+
+/* Model shape.  hidden must equal n_heads * head_dim; hidden and mlp_inner must be multiples of
+ * 8, head_dim even and <= 128.  dtype selects the storage type of weights, KV cache and GEMM
+ * inputs (accumulation, residual stream, latents, softmax and logits are always float32). */
+typedef struct {
+    int32_t hidden, n_heads, head_dim, mlp_inner;
+    int32_t n_prelude, n_core, n_coda, vocab;
+    int32_t dtype;          /* RD_F32 | RD_BF16 */
+    int32_t tie_embeddings; /* non-zero: the LM head is the embedding matrix */
+    float rope_base;        /* rotary base (10000) */
+    float norm_eps;         /* RMSNorm epsilon, added to the mean square */
+    float init_sigma;       /* sigma of s_0 ~ N(0, sigma^2 I) */
+} rd_config;
+
+typedef struct {
+    int32_t batch;             /* independent sequences stepped together                     */
+    int32_t max_context;       /* positions per sequence the KV caches hold                  */
+    int32_t max_window;        /* wavefront limiter: most in-flight positions per sequence   */
+    int32_t max_iters_per_pos; /* adaptive mode: core iterations after which a position is
+                                  treated as converged                                       */
+    int32_t max_new_tokens;    /* N of Algorithms 1-2, per sequence                          */
+    int32_t keep_logits;       /* non-zero: full logits of the last step stay readable       */
+    float temperature;         /* 0 => greedy (arg max, lowest index on ties); else Gumbel-max
+                                  sampling from softmax(logits / temperature)                */
+    uint64_t seed;             /* key of the counter-based generator (initial states, Gumbel) */
+} rd_session_config;
+
+typedef struct {
+    uint64_t df_steps, ar_steps;           /* calls that enqueued work                       */
+    uint64_t rows_prelude, rows_core, rows_coda; /* row-passes through P, R, C during decode
+                                              (cost remark of Section 3.5)                   */
+    uint64_t tokens_committed;             /* over all sequences, decode only                */
+    uint64_t kernel_launches;              /* kernels of this library launched so far        */
+    uint64_t tc_gemm_launches;             /* of those, tcgen05 GEMM launches                */
+} rd_stats_t;
+
+/* rd_load -- upload (or reference-free copy) of the weights of P, R, C (Section 3.1).
+ *   cfg           host pointer.
+ *   tensors       host array of pointers (each host or device memory), in this order:
+ *                 emb [V,h]; for block in prelude, core, coda, for each layer: g1 [h], wq [h,h],
+ *                 wk [h,h], wv [h,h], wo [h,h], g2 [h], wg [I,h], wu [I,h], wd [h,I];
+ *                 adapter [h,2h] (columns 0..h-1 multiply e, h..2h-1 multiply s); g_core [h];
+ *                 g_final [h]; head [V,h] only when tie_embeddings == 0.
+ *                 Gains (g*) are float32.  Matrices are float32 when elem_bytes == 4 and bfloat16
+ *                 bit patterns when elem_bytes == 2 (only valid with dtype RD_BF16); float32
+ *                 input with dtype RD_BF16 is rounded to nearest-even once.
+ *   n_tensors     length of `tensors` (checked against the shape).
+ *   out           receives the model.  Errors: INVALID_ARG, OOM, CUDA. */
+int rd_load(const rd_config* cfg, const void* const* tensors, int32_t n_tensors, int32_t elem_bytes,
+            rd_model** out);
+void rd_free(rd_model* m);
+
+/* rd_session_create -- allocate KV caches (three blocks, [layer][sequence][position][hidden]),
+ * latent slots and token arrays for `batch` sequences.
+ *   cuda_stream   a cudaStream_t (as void*) on which every step is enqueued; NULL = legacy
+ *                 default stream.  The model must outlive the session. */
+int rd_session_create(const rd_model* m, const rd_session_config* sc, void* cuda_stream,
+                      rd_session** out);
+void rd_session_destroy(rd_session* s);
+
+/* rd_prefill -- Section 3.3: positions 0..n_prompt-2 of sequence `seq` run P, `r` simultaneous
+ * passes of R (pass i of position p attends pass-i K/V of positions <= p) and the coda layers;
+ * position n_prompt-1 becomes the first in-flight position with a fresh state (Algorithm 1,
+ * lines 1-3).  prompt: host pointer to n_prompt token ids in [0, vocab).  Re-prefilling a
+ * sequence restarts it.  Errors: INVALID_ARG, CAPACITY (n_prompt + max_new_tokens >
+ * max_context), OOM, CUDA. */
+int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r);
+
+/* rd_ar_step -- one token on every live sequence by the sequential recurrence (Section 3.1):
+ * e = P(newest token), s_0, r applications of R, p = C(s_r), sample, commit.
+ * Errors: STATE (a sequence is not prefetched, or a wavefront wider than one is open). */
+int rd_ar_step(rd_session* s, int32_t r);
+
+/* rd_df_step -- one step of the diffusion-forcing sampler on every live sequence: e = P(y_current)
+ * on the in-flight rows, `inner_iters` applications of R, drafts from C for every row, freeze and
+ * commit the longest finished prefix, append one fresh position while fewer than `window` rows
+ * are in flight.  exit_threshold <= 0: fixed exit (Algorithm 1; a row is finished after `window`
+ * steps).  exit_threshold > 0: adaptive exit (Algorithm 2; finished when delta_i of Eq. 3 is below
+ * the threshold, or after max_iters_per_pos core iterations).  rd_df_step(1, r, 0) computes exactly
+ * what rd_ar_step(r) computes.  Errors: STATE, CAPACITY (window > max_window), INVALID_ARG. */
+int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, float exit_threshold);
+
+/* rd_sync -- wait for every enqueued step; returns TIMEOUT/CUDA if a kernel reported a fault. */
+int rd_sync(rd_session* s);
+
+/* rd_committed -- |y_frozen| of sequence `seq` (prompt + committed tokens); *done is set when the
+ * sequence has produced max_new_tokens.  Either out pointer may be NULL. */
+int rd_committed(rd_session* s, int32_t seq, int32_t* n_tokens, int32_t* done);
+
+/* rd_get_tokens -- copy up to `cap` tokens of y_frozen (prompt included) to host memory `dst`. */
+int rd_get_tokens(rd_session* s, int32_t seq, int32_t* dst, int32_t cap, int32_t* n_written);
+
+/* Inspection of the most recent step (rows are the positions that step processed, oldest first).
+ * rd_last_step_rows gives their first position and count; rd_debug_read copies to host `dst`:
+ *   RD_DBG_LATENTS float32 [n, hidden]   z after the step's last core iteration
+ *   RD_DBG_DELTA   float32 [n]           delta_i of Eq. 3 against the state at the step's start
+ *   RD_DBG_DRAFTS  int32   [n]           sampled tokens (row at position p drafts token p+1)
+ *   RD_DBG_LOGITS  float32 [n, vocab]    needs keep_logits
+ *   RD_DBG_EMBED   float32 [n, hidden]   e = P(y_current) of the step
+ * `bytes` must be at least the size above, else INVALID_ARG. */
+enum { RD_DBG_LATENTS = 0, RD_DBG_DELTA = 1, RD_DBG_DRAFTS = 2, RD_DBG_LOGITS = 3, RD_DBG_EMBED = 4 };
+int rd_last_step_rows(rd_session* s, int32_t seq, int32_t* first_pos, int32_t* n_rows);
+int rd_debug_read(rd_session* s, int32_t what, int32_t seq, void* dst, size_t bytes);
+
+/* rd_debug_force_tokens -- overwrite y_current[first_pos .. first_pos+n) (drafts or the newest
+ * committed tokens) from host memory; lets a lock-step comparison follow the other side through
+ * a near-tie.  Positions inside the prompt are refused (INVALID_ARG). */
+int rd_debug_force_tokens(rd_session* s, int32_t seq, int32_t first_pos, const int32_t* tokens,
+                          int32_t n);
+
+/* rd_debug_read_kv -- copy K (which=0) or V (which=1) of block (0 prelude, 1 core, 2 coda), layer,
+ * sequence, positions [pos0, pos0+n) to host `dst` as float32 [n, hidden]. */
+int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq,
+                     int32_t pos0, int32_t n, float* dst);
+
+/* rd_stats -- counters since session creation (host pointer out). */
+int rd_stats(rd_session* s, rd_stats_t* out);
+
+/* rd_set_gemm_path -- 0: SIMT kernels everywhere; 1 (default for RD_BF16): tcgen05 tensor-core
+ * GEMMs where the shape allows.  For measurement and parity tests. */
+int rd_set_gemm_path(rd_session* s, int32_t path);
+
+const char* rd_strerror(int code);
+/* Text of the last CUDA error this library saw on the calling thread's most recent failing call
+ * (static storage, never NULL). */
+const char* rd_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RD_H_ */

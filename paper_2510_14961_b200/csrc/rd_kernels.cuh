@@ -1,0 +1,455 @@
+// SIMT kernels of the recurrent-depth sampler: everything on the step that is not a tensor-core
+// GEMM (row planning, embedding, RMSNorm, rotary + KV write, attention, SwiGLU, sampling, the
+// convergence test of Eq. 3, the freeze/commit/advance logic of Algorithms 1-2), plus a plain
+// FFMA GEMM that serves the float32 configuration and acts as fallback for shapes the tensor-core
+// kernel does not take.  All reductions run in a fixed order: results are bit-reproducible.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace rd {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// 16-byte vector load of 16/sizeof(T) elements, widened to float.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    __device__ static __forceinline__ void load(const float* p, float* out) {
+        float4 v = *reinterpret_cast<const float4*>(p);
+        out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+    }
+};
+template <> struct Vec16<bf16> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ void load(const bf16* p, float* out) {
+        uint4 v = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            out[2 * i] = __uint_as_float(w[i] << 16);
+            out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+};
+
+// Sum over the block, same value in every thread; fixed order (xor tree, then warps 0..n-1).
+__device__ __forceinline__ float block_sum(float v, float* sm) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sm[w] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < nw; i++) t += sm[i];
+    return t;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11) and the two streams the method draws from.
+// Counter = (block, position, sequence, stream); key = the session seed.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+    for (int i = 0; i < 10; i++) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.x += 0x9E3779B9u;
+        k.y += 0xBB67AE85u;
+    }
+    return c;
+}
+enum { STREAM_INIT_STATE = 0, STREAM_GUMBEL = 1 };
+
+// u = ((x >> 9) + 1/2) 2^-23 lies in (0,1) and is exact in float32.
+__device__ __forceinline__ float unit_open(uint32_t x) { return ((float)(x >> 9) + 0.5f) * 1.1920928955078125e-07f; }
+
+// Row tables -----------------------------------------------------------------------------------
+// A "row" is one position being processed in this pass.  row_pos[i] < 0 marks an unused slot.
+
+// Decode: slot s = b*Wmax + (p mod Wmax) holds position p of sequence b while p is in flight.
+__global__ void plan_rows_kernel(const int* __restrict__ n_committed, const int* __restrict__ win_len,
+                                 const int* __restrict__ done, int B, int Wmax, int* __restrict__ row_pos,
+                                 int* __restrict__ row_seq, int* __restrict__ step_first,
+                                 int* __restrict__ step_n) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= B * Wmax) return;
+    const int b = s / Wmax, j = s % Wmax;
+    const int f = n_committed[b] - 1;
+    const int w = done[b] ? 0 : win_len[b];
+    const int p = f + ((j - f % Wmax + Wmax) % Wmax);
+    row_pos[s] = (p < f + w) ? p : -1;
+    row_seq[s] = b;
+    if (j == 0) { step_first[b] = f; step_n[b] = w; }
+}
+
+// Prefill: n consecutive positions of one sequence.
+__global__ void fill_rows_kernel(int seq, int start, int n, int n_slots, int* __restrict__ row_pos,
+                                 int* __restrict__ row_seq) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_slots) return;
+    row_pos[i] = i < n ? start + i : -1;
+    row_seq[i] = seq;
+}
+
+// s_0 ~ N(0, sigma^2 I), keyed by (seed, sequence, position): element j is output j%4 of block
+// j/4; the block's words x0..x3 give two Box-Muller pairs.  Evaluated in double (a few thousand
+// values per new row).  only_fresh: fill rows whose step counter is 0 (rows appended last step).
+__global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                                  const int* __restrict__ row_steps, int only_fresh, int hidden,
+                                  float sigma, uint64_t seed, float* __restrict__ z, size_t ldz) {
+    const int r = blockIdx.x;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    if (only_fresh && row_steps[r] != 0) return;
+    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const int nb = (hidden + 3) / 4;
+    for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
+        const uint4 x = philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, (uint32_t)row_seq[r], STREAM_INIT_STATE), key);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+        float out[4];
+#pragma unroll
+        for (int a = 0; a < 4; a += 2) {
+            const double u0 = ((double)(w[a] >> 9) + 0.5) * 1.1920928955078125e-07;
+            const double u1 = ((double)(w[a + 1] >> 9) + 0.5) * 1.1920928955078125e-07;
+            const double rad = sqrt(-2.0 * log(u0));
+            double sn, cs;
+            sincos(6.283185307179586476925286766559 * u1, &sn, &cs);
+            out[a] = (float)((double)sigma * (rad * cs));
+            out[a + 1] = (float)((double)sigma * (rad * sn));
+        }
+#pragma unroll
+        for (int a = 0; a < 4; a++)
+            if (blk * 4 + a < hidden) z[(size_t)r * ldz + blk * 4 + a] = out[a];
+    }
+}
+
+// x[row] = emb[token at the row's position]
+template <typename T>
+__global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                             const int* __restrict__ tokens, int tok_stride, const T* __restrict__ emb,
+                             int hidden, float* __restrict__ x) {
+    const int r = blockIdx.x;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    const int tok = tokens[(size_t)row_seq[r] * tok_stride + p];
+    for (int j = threadIdx.x; j < hidden; j += blockDim.x)
+        x[(size_t)r * hidden + j] = to_f(emb[(size_t)tok * hidden + j]);
+}
+
+// out[row] = g * x / sqrt(mean(x^2) + eps); one block per row.
+template <typename TO>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, size_t ldx, const float* __restrict__ g,
+                               int hidden, float eps, TO* __restrict__ out, size_t ldo,
+                               const int* __restrict__ row_pos) {
+    __shared__ float sm[32];
+    const int r = blockIdx.x;
+    if (row_pos && row_pos[r] < 0) return;
+    const float* xr = x + (size_t)r * ldx;
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < hidden; j += blockDim.x) ss += xr[j] * xr[j];
+    ss = block_sum(ss, sm);
+    const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
+    for (int j = threadIdx.x; j < hidden; j += blockDim.x)
+        out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xr[j] * inv));
+}
+
+// act[row] = [ e[row] ; z[row] ] in the GEMM input type (adapter input, Section 3.2).
+template <typename T>
+__global__ void concat_kernel(const float* __restrict__ e, size_t lde, const float* __restrict__ z,
+                              size_t ldz, int hidden, T* __restrict__ act, size_t lda,
+                              const int* __restrict__ row_pos) {
+    const int r = blockIdx.x;
+    if (row_pos[r] < 0) return;
+    for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
+        act[(size_t)r * lda + j] = from_f<T>(e[(size_t)r * lde + j]);
+        act[(size_t)r * lda + hidden + j] = from_f<T>(z[(size_t)r * ldz + j]);
+    }
+}
+
+// Plain GEMM  Y[r, o] = sum_k A[r, k] W[o, k] (+ resid[r, o]);  one warp per output feature,
+// RT rows per warp, 16-byte loads, lanes split K, xor-tree reduction.
+template <typename T, int RT>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const T* __restrict__ A, size_t lda, const T* __restrict__ W, int K, int n_out,
+                 float* __restrict__ Y, size_t ldy, const float* __restrict__ resid, size_t ldr, int n_rows) {
+    constexpr int VEC = Vec16<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int r0 = blockIdx.y * RT;
+    if (o >= n_out) return;
+    float acc[RT];
+#pragma unroll
+    for (int r = 0; r < RT; r++) acc[r] = 0.f;
+    const T* wrow = W + (size_t)o * K;
+    for (int k = lane * VEC; k < K; k += 32 * VEC) {
+        float wf[VEC];
+        Vec16<T>::load(wrow + k, wf);
+#pragma unroll
+        for (int r = 0; r < RT; r++) {
+            const int rr = min(r0 + r, n_rows - 1);
+            float af[VEC];
+            Vec16<T>::load(A + (size_t)rr * lda + k, af);
+#pragma unroll
+            for (int i = 0; i < VEC; i++) acc[r] = fmaf(af[i], wf[i], acc[r]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < RT; r++) {
+        float v = acc[r];
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+        if (lane == 0 && r0 + r < n_rows) {
+            const size_t row = (size_t)(r0 + r);
+            Y[row * ldy + o] = resid ? resid[row * ldr + o] + v : v;
+        }
+    }
+}
+
+// Rotary embedding on adjacent pairs of q and k, then: q -> q_t (GEMM/attention input type),
+// k, v -> the row's own cache entry (overwrite: KV-cache sharing, Section 3.2).
+// qkv: [rows, 3h] float32 (q | k | v).  cos/sin: [max_ctx, d/2] float32.
+template <typename T>
+__global__ void rope_kv_kernel(const float* __restrict__ qkv, const int* __restrict__ row_pos,
+                               const int* __restrict__ row_seq, const float* __restrict__ cos_t,
+                               const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
+                               T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride) {
+    const int r = blockIdx.x;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    const int half = head_dim / 2;
+    const float* src = qkv + (size_t)r * 3 * hidden;
+    T* kdst = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
+    T* vdst = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
+    for (int idx = threadIdx.x; idx < hidden / 2; idx += blockDim.x) {
+        const int i = idx % half;
+        const float c = cos_t[(size_t)p * half + i], s = sin_t[(size_t)p * half + i];
+        const float q0 = src[2 * idx], q1 = src[2 * idx + 1];
+        const float k0 = src[hidden + 2 * idx], k1 = src[hidden + 2 * idx + 1];
+        q_t[(size_t)r * hidden + 2 * idx] = from_f<T>(q0 * c - q1 * s);
+        q_t[(size_t)r * hidden + 2 * idx + 1] = from_f<T>(q0 * s + q1 * c);
+        kdst[2 * idx] = from_f<T>(k0 * c - k1 * s);
+        kdst[2 * idx + 1] = from_f<T>(k0 * s + k1 * c);
+        vdst[2 * idx] = from_f<T>(src[2 * hidden + 2 * idx]);
+        vdst[2 * idx + 1] = from_f<T>(src[2 * hidden + 2 * idx + 1]);
+    }
+}
+
+// Causal attention, one block (4 warps) per (row, head): the row at position p attends cache
+// entries 0..p of its sequence (committed prefix, and in-flight rows <= p as written this pass).
+// Warps take keys round-robin with an online softmax; partials merge in warp order.
+template <typename T>
+__global__ void __launch_bounds__(128)
+attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                const T* __restrict__ Kc, const T* __restrict__ Vc, size_t seq_stride, int hidden,
+                int head_dim, float scale, T* __restrict__ out) {
+    __shared__ float sm_m[4], sm_l[4], sm_o[4][128];
+    const int r = blockIdx.x, hd = blockIdx.y;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const T* kb = Kc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_dim;
+    const T* vb = Vc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_dim;
+    float q[4], o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int t = 0; t < 4; t++) {
+        const int e = lane + 32 * t;
+        q[t] = e < head_dim ? to_f(q_t[(size_t)r * hidden + hd * head_dim + e]) : 0.f;
+    }
+    float m = -INFINITY, l = 0.f;
+    for (int j = warp; j <= p; j += 4) {
+        float d = 0.f;
+#pragma unroll
+        for (int t = 0; t < 4; t++) {
+            const int e = lane + 32 * t;
+            if (e < head_dim) d = fmaf(q[t], to_f(kb[(size_t)j * hidden + e]), d);
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
+        d *= scale;
+        const float mn = fmaxf(m, d);
+        const float corr = expf(m - mn), pj = expf(d - mn);
+        l = l * corr + pj;
+#pragma unroll
+        for (int t = 0; t < 4; t++) {
+            const int e = lane + 32 * t;
+            if (e < head_dim) o[t] = o[t] * corr + pj * to_f(vb[(size_t)j * hidden + e]);
+        }
+        m = mn;
+    }
+    if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+#pragma unroll
+    for (int t = 0; t < 4; t++) sm_o[warp][lane + 32 * t] = o[t];
+    __syncthreads();
+    if (warp == 0) {
+        float mm = sm_m[0];
+        for (int w = 1; w < 4; w++) mm = fmaxf(mm, sm_m[w]);
+        float ll = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int w = 0; w < 4; w++) {
+            if (sm_m[w] == -INFINITY) continue;      // warp saw no key
+            const float c = expf(sm_m[w] - mm);
+            ll += sm_l[w] * c;
+#pragma unroll
+            for (int t = 0; t < 4; t++) acc[t] += sm_o[w][lane + 32 * t] * c;
+        }
+#pragma unroll
+        for (int t = 0; t < 4; t++) {
+            const int e = lane + 32 * t;
+            if (e < head_dim) out[(size_t)r * hidden + hd * head_dim + e] = from_f<T>(acc[t] / ll);
+        }
+    }
+}
+
+// act[r, j] = silu(gu[r, j]) * gu[r, I + j]
+template <typename T>
+__global__ void swiglu_kernel(const float* __restrict__ gu, int inner, T* __restrict__ act, size_t lda,
+                              int n_rows) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)n_rows * inner) return;
+    const size_t r = i / inner, j = i % inner;
+    const float g = gu[r * 2 * inner + j], u = gu[r * 2 * inner + inner + j];
+    act[r * lda + j] = from_f<T>((g / (1.0f + expf(-g))) * u);
+}
+
+// Sample(p) of Algorithms 1-2, one block per row.  Greedy: arg max, lowest index on ties.
+// Otherwise Gumbel-max: arg max of logit / T - log(-log u_v), u_v keyed by (seed, sequence,
+// token position, v).  The row at position p drafts the token of position p + 1.
+__global__ void __launch_bounds__(256)
+sample_kernel(const float* __restrict__ logits, int vocab, const int* __restrict__ row_pos,
+              const int* __restrict__ row_seq, float temperature, uint64_t seed, int* __restrict__ draft,
+              int* __restrict__ tokens, int tok_stride) {
+    __shared__ float sv[8];
+    __shared__ int si[8];
+    const int r = blockIdx.x;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    const float* lg = logits + (size_t)r * vocab;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    if (temperature <= 0.f) {
+        for (int v = threadIdx.x; v < vocab; v += blockDim.x) {
+            const float x = lg[v];
+            if (x > best) { best = x; bi = v; }
+        }
+    } else {
+        const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+        const int nb = (vocab + 3) / 4;
+        for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
+            const uint4 x = philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)(p + 1), (uint32_t)row_seq[r], STREAM_GUMBEL), key);
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int a = 0; a < 4; a++) {
+                const int v = blk * 4 + a;
+                if (v < vocab) {
+                    const float g = -logf(-logf(unit_open(w[a])));
+                    const float sc = __fadd_rn(__fdiv_rn(lg[v], temperature), g);
+                    if (sc > best) { best = sc; bi = v; }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, s);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); w++)
+            if (sv[w] > best || (sv[w] == best && si[w] < bi)) { best = sv[w]; bi = si[w]; }
+        if (bi == 0x7fffffff) bi = 0;                 // all -inf / NaN row: defined result
+        draft[r] = bi;
+        tokens[(size_t)row_seq[r] * tok_stride + p + 1] = bi;
+    }
+}
+
+// delta_i = ||z_i - z_prev,i|| / ||z_i||  (Eq. 3); +inf when ||z_i|| = 0.
+__global__ void __launch_bounds__(256)
+delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int hidden,
+             const int* __restrict__ row_pos, float* __restrict__ delta) {
+    __shared__ float sm[32];
+    const int r = blockIdx.x;
+    if (row_pos[r] < 0) return;
+    float num = 0.f, den = 0.f;
+    for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
+        const float a = z[(size_t)r * hidden + j], d = a - z_prev[(size_t)r * hidden + j];
+        num += d * d;
+        den += a * a;
+    }
+    num = block_sum(num, sm);
+    den = block_sum(den, sm);
+    if (threadIdx.x == 0) delta[r] = den > 0.f ? sqrtf(num) / sqrtf(den) : INFINITY;
+}
+
+// End of a step, one thread per sequence: count the step on every in-flight row, find k* (the
+// longest finished prefix; Eq. 3 / Algorithm 1 line 14), commit, drop, append one fresh row while
+// the wavefront is below `window` and the row's draft is still wanted.
+struct SeqState {
+    int* n_prompt; int* n_committed; int* win_len; int* done;
+    int* row_steps; int* row_iters;
+    unsigned long long* counters;   // [0] rows through P, [1] R, [2] C, [3] tokens committed
+};
+__global__ void advance_kernel(SeqState st, const float* __restrict__ delta, int B, int Wmax, int window,
+                               int inner_iters, float exit_threshold, int cap, int max_new) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B || st.done[b]) return;
+    const int f = st.n_committed[b] - 1;
+    int w = st.win_len[b];
+    int k = 0;
+    bool open = true;
+    for (int i = 0; i < w; i++) {
+        const int s = b * Wmax + (f + i) % Wmax;
+        const int steps = ++st.row_steps[s];
+        const int iters = (st.row_iters[s] += inner_iters);
+        const bool fin = exit_threshold <= 0.f ? steps >= window : (delta[s] < exit_threshold || iters >= cap);
+        if (open && fin) k++; else open = false;
+    }
+    atomicAdd(&st.counters[0], (unsigned long long)w);
+    atomicAdd(&st.counters[1], (unsigned long long)w * inner_iters);
+    atomicAdd(&st.counters[2], (unsigned long long)w);
+    int nc = st.n_committed[b];
+    const int np = st.n_prompt[b];
+    k = min(k, max_new - (nc - np));
+    nc += k;
+    w -= k;
+    atomicAdd(&st.counters[3], (unsigned long long)k);
+    if (nc - np >= max_new) {
+        st.done[b] = 1;
+        w = 0;
+    } else if (w < window) {
+        const int nxt = nc - 1 + w;
+        if (nxt <= np + max_new - 2) {
+            const int s = b * Wmax + nxt % Wmax;
+            st.row_steps[s] = 0;
+            st.row_iters[s] = 0;
+            w++;
+        }
+    }
+    st.n_committed[b] = nc;
+    st.win_len[b] = w;
+}
+
+// float32 -> T copy (weight upload path; bf16 rounds to nearest even once).
+template <typename T>
+__global__ void convert_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = from_f<T>(src[i]);
+}
+template <typename T>
+__global__ void widen_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = to_f(src[i]);
+}
+
+}  // namespace rd

@@ -1,0 +1,683 @@
+// Host side of the C ABI declared in include/rd.h: model and session objects, the schedule of one
+// prefill / AR step / diffusion-forcing step, and the inspection calls.  Every arithmetic step of
+// the path runs in the kernels of rd_kernels.cuh and rd_gemm_tc.cuh; this file only launches them.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "../../include/rd.h"
+#include "rd_gemm_tc.cuh"
+#include "rd_kernels.cuh"
+
+using namespace rd;
+
+// ---------------------------------------------------------------------------------------------
+// Error plumbing
+// ---------------------------------------------------------------------------------------------
+static thread_local char g_cuda_err[320] = "no CUDA error recorded";
+
+static int cuda_fail(cudaError_t e, const char* what, int line) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s (%s) at rd_lib.cu:%d: %s", cudaGetErrorName(e), what, line,
+             cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? RD_E_OOM : RD_E_CUDA;
+}
+#define CU(expr)                                                        \
+    do {                                                                \
+        cudaError_t e_ = (expr);                                        \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #expr, __LINE__);   \
+    } while (0)
+#define RD_TRY(expr)                 \
+    do {                             \
+        int rc_ = (expr);            \
+        if (rc_ != RD_OK) return rc_; \
+    } while (0)
+
+extern "C" const char* rd_last_cuda_error(void) { return g_cuda_err; }
+extern "C" const char* rd_strerror(int code) {
+    switch (code) {
+        case RD_OK: return "ok";
+        case RD_E_INVALID_ARG: return "invalid argument";
+        case RD_E_STATE: return "call out of order for the session's state";
+        case RD_E_CAPACITY: return "capacity exceeded (context or window)";
+        case RD_E_OOM: return "out of device memory";
+        case RD_E_CUDA: return "CUDA error";
+        case RD_E_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error code";
+    }
+}
+
+// Device allocations owned by one object; zero-filled; freed together.
+struct DevMem {
+    std::vector<void*> ptrs;
+    template <typename P> int get(P** out, size_t bytes) {
+        void* p = nullptr;
+        if (bytes == 0) bytes = 16;
+        cudaError_t e = cudaMalloc(&p, bytes);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc", __LINE__);
+        e = cudaMemset(p, 0, bytes);
+        if (e != cudaSuccess) { cudaFree(p); return cuda_fail(e, "cudaMemset", __LINE__); }
+        ptrs.push_back(p);
+        *out = reinterpret_cast<P*>(p);
+        return RD_OK;
+    }
+    void release(void* p) {
+        for (size_t i = 0; i < ptrs.size(); i++)
+            if (ptrs[i] == p) { cudaFree(p); ptrs.erase(ptrs.begin() + i); return; }
+    }
+    ~DevMem() { for (void* p : ptrs) cudaFree(p); }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Model
+// ---------------------------------------------------------------------------------------------
+struct LayerW {
+    float* g1 = nullptr; void* wqkv = nullptr; void* wo = nullptr;
+    float* g2 = nullptr; void* wgu = nullptr; void* wd = nullptr;
+    TcWeight t_qkv, t_o, t_gu, t_d;
+};
+
+struct rd_model {
+    rd_config cfg;
+    int device = 0;
+    size_t esz = 4;
+    DevMem mem;
+    void* emb = nullptr; void* head = nullptr; void* adapter = nullptr;
+    float* g_core = nullptr; float* g_final = nullptr;
+    std::vector<LayerW> layers[3];
+    TcWeight t_adapter, t_head;
+    bool tc_ok = false;
+};
+
+static int n_layers_of(const rd_config& c, int blk) { return blk == 0 ? c.n_prelude : blk == 1 ? c.n_core : c.n_coda; }
+
+// Copy one source tensor (host or device memory) into `dst`, converting float32 -> bf16 on the
+// device when the model stores bf16.
+static int put_tensor(rd_model* m, void* dst, const void* src, size_t n, int elem_bytes, float** stage,
+                      size_t* stage_n) {
+    if (m->esz == (size_t)elem_bytes) {
+        CU(cudaMemcpy(dst, src, n * m->esz, cudaMemcpyDefault));
+        return RD_OK;
+    }
+    if (*stage_n < n) {
+        if (*stage) { cudaFree(*stage); *stage = nullptr; *stage_n = 0; }
+        CU(cudaMalloc((void**)stage, n * sizeof(float)));
+        *stage_n = n;
+    }
+    CU(cudaMemcpy(*stage, src, n * sizeof(float), cudaMemcpyDefault));
+    convert_kernel<bf16><<<1024, 256>>>(*stage, (bf16*)dst, n);
+    CU(cudaGetLastError());
+    CU(cudaDeviceSynchronize());
+    return RD_OK;
+}
+
+static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
+    const rd_config& c = m->cfg;
+    const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
+    float* stage = nullptr;
+    size_t stage_n = 0;
+    int rc = RD_OK;
+    int idx = 0;
+    auto mat = [&](void* dst, size_t n) -> int { return put_tensor(m, dst, t[idx++], n, elem_bytes, &stage, &stage_n); };
+    auto gain = [&](float** dst) -> int {
+        RD_TRY(m->mem.get(dst, h * sizeof(float)));
+        CU(cudaMemcpy(*dst, t[idx++], h * sizeof(float), cudaMemcpyDefault));
+        return RD_OK;
+    };
+    do {
+        if ((rc = m->mem.get(&m->emb, V * h * es))) break;
+        if ((rc = mat(m->emb, V * h))) break;
+        for (int blk = 0; blk < 3 && !rc; blk++) {
+            m->layers[blk].resize(n_layers_of(c, blk));
+            for (LayerW& L : m->layers[blk]) {
+                if ((rc = gain(&L.g1))) break;
+                if ((rc = m->mem.get(&L.wqkv, 3 * h * h * es))) break;
+                for (int j = 0; j < 3 && !rc; j++) rc = mat((char*)L.wqkv + j * h * h * es, h * h);
+                if (rc) break;
+                if ((rc = m->mem.get(&L.wo, h * h * es))) break;
+                if ((rc = mat(L.wo, h * h))) break;
+                if ((rc = gain(&L.g2))) break;
+                if ((rc = m->mem.get(&L.wgu, 2 * I * h * es))) break;
+                if ((rc = mat(L.wgu, I * h))) break;
+                if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
+                if ((rc = m->mem.get(&L.wd, h * I * es))) break;
+                if ((rc = mat(L.wd, h * I))) break;
+            }
+        }
+        if (rc) break;
+        if ((rc = m->mem.get(&m->adapter, 2 * h * h * es))) break;
+        if ((rc = mat(m->adapter, 2 * h * h))) break;
+        if ((rc = gain(&m->g_core))) break;
+        if ((rc = gain(&m->g_final))) break;
+        if (c.tie_embeddings) {
+            m->head = m->emb;
+        } else {
+            if ((rc = m->mem.get(&m->head, V * h * es))) break;
+            if ((rc = mat(m->head, V * h))) break;
+        }
+    } while (0);
+    if (stage) cudaFree(stage);
+    if (rc) return rc;
+    // Tensor-core path: TMA descriptors over every weight matrix (bf16 only).
+    m->tc_ok = false;
+    if (c.dtype == RD_BF16 && tc_init_driver() == RD_OK) {
+        bool ok = true;
+        for (int blk = 0; blk < 3; blk++)
+            for (LayerW& L : m->layers[blk]) {
+                ok &= tc_make_weight(&L.t_qkv, L.wqkv, 3 * c.hidden, c.hidden) == RD_OK;
+                ok &= tc_make_weight(&L.t_o, L.wo, c.hidden, c.hidden) == RD_OK;
+                ok &= tc_make_weight(&L.t_gu, L.wgu, 2 * c.mlp_inner, c.hidden) == RD_OK;
+                ok &= tc_make_weight(&L.t_d, L.wd, c.hidden, c.mlp_inner) == RD_OK;
+            }
+        ok &= tc_make_weight(&m->t_adapter, m->adapter, c.hidden, 2 * c.hidden) == RD_OK;
+        ok &= tc_make_weight(&m->t_head, m->head, c.vocab, c.hidden) == RD_OK;
+        m->tc_ok = ok;
+    }
+    return RD_OK;
+}
+
+extern "C" int rd_load(const rd_config* cfg, const void* const* tensors, int32_t n_tensors, int32_t elem_bytes,
+                       rd_model** out) {
+    if (!cfg || !tensors || !out) return RD_E_INVALID_ARG;
+    const rd_config& c = *cfg;
+    if (c.hidden <= 0 || c.n_heads <= 0 || c.head_dim <= 0 || c.mlp_inner <= 0 || c.vocab <= 0) return RD_E_INVALID_ARG;
+    if (c.hidden != c.n_heads * c.head_dim || c.hidden % 8 || c.mlp_inner % 8) return RD_E_INVALID_ARG;
+    if (c.head_dim % 2 || c.head_dim > 128) return RD_E_INVALID_ARG;
+    if (c.n_prelude < 0 || c.n_core < 1 || c.n_coda < 0) return RD_E_INVALID_ARG;
+    if (c.dtype != RD_F32 && c.dtype != RD_BF16) return RD_E_INVALID_ARG;
+    if (elem_bytes != 4 && !(elem_bytes == 2 && c.dtype == RD_BF16)) return RD_E_INVALID_ARG;
+    if (!(c.norm_eps >= 0.f) || !(c.rope_base > 0.f) || !(c.init_sigma >= 0.f)) return RD_E_INVALID_ARG;
+    const int want = 1 + 9 * (c.n_prelude + c.n_core + c.n_coda) + 3 + (c.tie_embeddings ? 0 : 1);
+    if (n_tensors != want) return RD_E_INVALID_ARG;
+    for (int i = 0; i < n_tensors; i++)
+        if (!tensors[i]) return RD_E_INVALID_ARG;
+    rd_model* m = new (std::nothrow) rd_model();
+    if (!m) return RD_E_OOM;
+    m->cfg = c;
+    m->esz = c.dtype == RD_BF16 ? 2 : 4;
+    cudaError_t e = cudaGetDevice(&m->device);
+    if (e != cudaSuccess) { delete m; return cuda_fail(e, "cudaGetDevice", __LINE__); }
+    const int rc = load_impl(m, tensors, elem_bytes);
+    if (rc) { delete m; return rc; }
+    *out = m;
+    return RD_OK;
+}
+extern "C" void rd_free(rd_model* m) { delete m; }
+
+// ---------------------------------------------------------------------------------------------
+// Session
+// ---------------------------------------------------------------------------------------------
+struct rd_session {
+    const rd_model* m = nullptr;
+    rd_session_config sc;
+    cudaStream_t stream = nullptr;
+    DevMem mem;
+    int n_slots = 0;   // batch * max_window: decode rows
+    int R = 0;         // row capacity of the scratch buffers (>= n_slots; prefill chunk size)
+    int tok_stride = 0;
+    size_t seq_stride = 0;   // elements between sequences in a cache layer
+    // device state
+    int *tokens = nullptr, *n_prompt = nullptr, *n_committed = nullptr, *win_len = nullptr, *done = nullptr;
+    int *row_steps = nullptr, *row_iters = nullptr, *row_pos = nullptr, *row_seq = nullptr;
+    int *step_first = nullptr, *step_n = nullptr, *draft = nullptr;
+    unsigned long long* counters = nullptr;
+    int* status = nullptr;   // device word: non-zero when a bounded wait ran out
+    float *x = nullptr, *qkv = nullptr, *gu = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
+    float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
+    float* partial = nullptr;   // split-K partial sums of the tensor-core GEMM
+    size_t partial_elems = 0;
+    void *act_h = nullptr, *act_2h = nullptr, *act_i = nullptr, *q_t = nullptr;
+    void *Kc[3] = {nullptr, nullptr, nullptr}, *Vc[3] = {nullptr, nullptr, nullptr};
+    TcAct t_act_h, t_act_2h, t_act_i;
+    // host state
+    std::vector<char> prefilled, wave_open;
+    int gemm_path = 0;
+    rd_stats_t stats;
+};
+
+#define LAUNCHED(s)                  \
+    do {                             \
+        (s)->stats.kernel_launches++; \
+        CU(cudaGetLastError());      \
+    } while (0)
+
+extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp, void* cuda_stream,
+                                 rd_session** out) {
+    if (!m || !scp || !out) return RD_E_INVALID_ARG;
+    const rd_session_config& sc = *scp;
+    if (sc.batch < 1 || sc.max_context < 2 || sc.max_window < 1 || sc.max_new_tokens < 0) return RD_E_INVALID_ARG;
+    if (sc.max_iters_per_pos < 1 || !(sc.temperature >= 0.f)) return RD_E_INVALID_ARG;
+    if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
+    rd_session* s = new (std::nothrow) rd_session();
+    if (!s) return RD_E_OOM;
+    s->m = m;
+    s->sc = sc;
+    s->stream = (cudaStream_t)cuda_stream;
+    memset(&s->stats, 0, sizeof s->stats);
+    const rd_config& c = m->cfg;
+    const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
+    s->n_slots = sc.batch * sc.max_window;
+    s->R = std::max(s->n_slots, 128);
+    s->R = (s->R + 15) / 16 * 16;
+    s->tok_stride = sc.max_context + 1;
+    s->seq_stride = (size_t)sc.max_context * h;
+    const size_t R = s->R, B = sc.batch;
+    int rc = RD_OK;
+    do {
+        if ((rc = s->mem.get(&s->tokens, B * s->tok_stride * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->n_prompt, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->n_committed, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->win_len, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->done, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->step_first, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->step_n, B * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->row_steps, R * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->row_iters, R * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->row_pos, R * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->row_seq, R * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->draft, R * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->counters, 8 * sizeof(unsigned long long)))) break;
+        if ((rc = s->mem.get(&s->status, 4 * sizeof(int)))) break;
+        if ((rc = s->mem.get(&s->x, R * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->qkv, R * 3 * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->gu, R * 2 * I * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->e, R * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->z, R * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->z_prev, R * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->logits, (size_t)s->n_slots * V * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->delta, R * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->act_h, R * h * es))) break;
+        if ((rc = s->mem.get(&s->act_2h, R * 2 * h * es))) break;
+        if ((rc = s->mem.get(&s->act_i, R * I * es))) break;
+        if ((rc = s->mem.get(&s->q_t, R * h * es))) break;
+        for (int blk = 0; blk < 3 && !rc; blk++) {
+            const size_t n = (size_t)n_layers_of(c, blk) * B * s->seq_stride * es;
+            if ((rc = s->mem.get(&s->Kc[blk], n))) break;
+            rc = s->mem.get(&s->Vc[blk], n);
+        }
+        if (rc) break;
+        // Rotary tables: angle pos * base^(-2i/d), evaluated in double, stored as float32.
+        const int half = c.head_dim / 2;
+        std::vector<float> ct((size_t)sc.max_context * half), st((size_t)sc.max_context * half);
+        for (int p = 0; p < sc.max_context; p++)
+            for (int i = 0; i < half; i++) {
+                const double ang = (double)p * pow((double)c.rope_base, -2.0 * i / c.head_dim);
+                ct[(size_t)p * half + i] = (float)cos(ang);
+                st[(size_t)p * half + i] = (float)sin(ang);
+            }
+        if ((rc = s->mem.get(&s->cos_t, ct.size() * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->sin_t, st.size() * sizeof(float)))) break;
+        cudaError_t e = cudaMemcpy(s->cos_t, ct.data(), ct.size() * sizeof(float), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(s->sin_t, st.data(), st.size() * sizeof(float), cudaMemcpyHostToDevice);
+        // every sequence starts "done" until it is prefilled
+        std::vector<int> ones(B, 1);
+        if (e == cudaSuccess) e = cudaMemcpy(s->done, ones.data(), B * sizeof(int), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { rc = cuda_fail(e, "session init copies", __LINE__); break; }
+        if (m->tc_ok) {
+            s->partial_elems = tc_partial_elems(R, c);
+            if ((rc = s->mem.get(&s->partial, s->partial_elems * sizeof(float)))) break;
+            bool ok = tc_make_act(&s->t_act_h, s->act_h, s->R, c.hidden) == RD_OK;
+            ok &= tc_make_act(&s->t_act_2h, s->act_2h, s->R, 2 * c.hidden) == RD_OK;
+            ok &= tc_make_act(&s->t_act_i, s->act_i, s->R, c.mlp_inner) == RD_OK;
+            s->gemm_path = ok ? 1 : 0;
+        }
+    } while (0);
+    if (rc) { delete s; return rc; }
+    s->prefilled.assign(B, 0);
+    s->wave_open.assign(B, 0);
+    *out = s;
+    return RD_OK;
+}
+extern "C" void rd_session_destroy(rd_session* s) {
+    if (!s) return;
+    cudaStreamSynchronize(s->stream);
+    delete s;
+}
+extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
+    if (!s || (path != 0 && path != 1)) return RD_E_INVALID_ARG;
+    if (path == 1 && !(s->m->tc_ok && s->partial)) return RD_E_STATE;
+    s->gemm_path = path;
+    return RD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The schedule (templated on the storage type T of weights / KV / GEMM inputs)
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Eng {
+    // Y[r, o] = sum_k A[r, k] W[o, k] (+ resid).  `ta`/`tw` are the operands' TMA descriptors for
+    // the tensor-core path (bf16 only).
+    static int gemm(rd_session* s, const T* A, size_t lda, const TcAct* ta, const T* W, const TcWeight* tw, int K,
+                    int n_out, float* Y, size_t ldy, const float* resid, int n_rows) {
+        if (sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid) {
+            const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, Y, ldy, resid, n_rows, s->partial,
+                                   s->partial_elems, s->status, &s->stats.kernel_launches);
+            if (rc == RD_OK) { s->stats.tc_gemm_launches++; return RD_OK; }
+            if (rc != RD_E_INVALID_ARG) return rc;   // INVALID_ARG: shape not taken, fall through
+        }
+        const int warps = 8;
+        dim3 grid((n_out + warps - 1) / warps, 1);
+        if (n_rows == 1) {
+            gemm_simt_kernel<T, 1><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+        } else if (n_rows <= 4) {
+            gemm_simt_kernel<T, 4><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+        } else {
+            grid.y = (n_rows + 7) / 8;
+            gemm_simt_kernel<T, 8><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+        }
+        LAUNCHED(s);
+        return RD_OK;
+    }
+
+    // One transformer layer over the rows of the current row table, in place on x.
+    static int layer(rd_session* s, int blk, int l, float* x, int n_rows) {
+        const rd_config& c = s->m->cfg;
+        const LayerW& L = s->m->layers[blk][l];
+        const int h = c.hidden, I = c.mlp_inner;
+        const size_t layer_off = (size_t)l * s->sc.batch * s->seq_stride;
+        T* Kc = (T*)s->Kc[blk] + layer_off;
+        T* Vc = (T*)s->Vc[blk] + layer_off;
+        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g1, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, s->qkv, 3 * h, nullptr, n_rows));
+        rope_kv_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->qkv, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h,
+                                                          c.head_dim, (T*)s->q_t, Kc, Vc, s->seq_stride);
+        LAUNCHED(s);
+        attn_row_kernel<T><<<dim3(n_rows, c.n_heads), 128, 0, s->stream>>>(
+            (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc, s->seq_stride, h, c.head_dim,
+            (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, x, h, x, n_rows));
+        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g2, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, s->gu, 2 * I, nullptr, n_rows));
+        const size_t n_el = (size_t)n_rows * I;
+        swiglu_kernel<T><<<(unsigned)((n_el + 255) / 256), 256, 0, s->stream>>>(s->gu, I, (T*)s->act_i, I, n_rows);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, x, h, x, n_rows));
+        return RD_OK;
+    }
+
+    // e = P(tokens of the rows): embedding + prelude layers; result left in s->x.
+    static int prelude(rd_session* s, int n_rows) {
+        const rd_config& c = s->m->cfg;
+        embed_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->row_pos, s->row_seq, s->tokens, s->tok_stride,
+                                                        (const T*)s->m->emb, c.hidden, s->x);
+        LAUNCHED(s);
+        for (int l = 0; l < c.n_prelude; l++) RD_TRY(layer(s, 0, l, s->x, n_rows));
+        return RD_OK;
+    }
+
+    // z_out = R(e, z_in): adapter over concat(e, z), core layers, closing RMSNorm.
+    static int core(rd_session* s, const float* e, const float* z_in, float* z_out, int n_rows) {
+        const rd_config& c = s->m->cfg;
+        const int h = c.hidden;
+        concat_kernel<T><<<n_rows, 256, 0, s->stream>>>(e, h, z_in, h, h, (T*)s->act_2h, 2 * h, s->row_pos);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, s->x, h,
+                    nullptr, n_rows));
+        for (int l = 0; l < c.n_core; l++) RD_TRY(layer(s, 1, l, s->x, n_rows));
+        rmsnorm_kernel<float><<<n_rows, 256, 0, s->stream>>>(s->x, h, s->m->g_core, h, c.norm_eps, z_out, h, s->row_pos);
+        LAUNCHED(s);
+        return RD_OK;
+    }
+
+    // Coda layers on x = z; with `head`: final RMSNorm, LM head, Sample -> drafts.
+    static int coda(rd_session* s, const float* z, int n_rows, bool head) {
+        const rd_config& c = s->m->cfg;
+        const int h = c.hidden;
+        CU(cudaMemcpyAsync(s->x, z, (size_t)n_rows * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+        for (int l = 0; l < c.n_coda; l++) RD_TRY(layer(s, 2, l, s->x, n_rows));
+        if (!head) return RD_OK;
+        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->x, h, s->m->g_final, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
+        LAUNCHED(s);
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, s->logits, c.vocab,
+                    nullptr, n_rows));
+        sample_kernel<<<n_rows, 256, 0, s->stream>>>(s->logits, c.vocab, s->row_pos, s->row_seq, s->sc.temperature,
+                                                     s->sc.seed, s->draft, s->tokens, s->tok_stride);
+        LAUNCHED(s);
+        return RD_OK;
+    }
+
+    // One sampler step over the decode slots (Algorithm 1 / Algorithm 2; AR is window 1).
+    static int decode_step(rd_session* s, int window, int inner, float eps) {
+        const rd_config& c = s->m->cfg;
+        const int n = s->n_slots, h = c.hidden, B = s->sc.batch;
+        plan_rows_kernel<<<(n + 127) / 128, 128, 0, s->stream>>>(s->n_committed, s->win_len, s->done, B,
+                                                                 s->sc.max_window, s->row_pos, s->row_seq,
+                                                                 s->step_first, s->step_n);
+        LAUNCHED(s);
+        init_state_kernel<<<n, 128, 0, s->stream>>>(s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma,
+                                                    s->sc.seed, s->z, h);
+        LAUNCHED(s);
+        CU(cudaMemcpyAsync(s->z_prev, s->z, (size_t)n * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+        RD_TRY(prelude(s, n));
+        CU(cudaMemcpyAsync(s->e, s->x, (size_t)n * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+        for (int j = 0; j < inner; j++) RD_TRY(core(s, s->e, s->z, s->z, n));
+        RD_TRY(coda(s, s->z, n, true));
+        delta_kernel<<<n, 256, 0, s->stream>>>(s->z, s->z_prev, h, s->row_pos, s->delta);
+        LAUNCHED(s);
+        SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
+        advance_kernel<<<(B + 63) / 64, 64, 0, s->stream>>>(st, s->delta, B, s->sc.max_window, window, inner, eps,
+                                                            s->sc.max_iters_per_pos, s->sc.max_new_tokens);
+        LAUNCHED(s);
+        return RD_OK;
+    }
+
+    static int prefill(rd_session* s, int seq, const int32_t* prompt, int L, int r) {
+        const rd_config& c = s->m->cfg;
+        const int h = c.hidden;
+        CU(cudaStreamSynchronize(s->stream));
+        CU(cudaMemcpy(s->tokens + (size_t)seq * s->tok_stride, prompt, (size_t)L * sizeof(int), cudaMemcpyHostToDevice));
+        const int n = L - 1;   // rows 0..L-2 are prefilled; L-1 is the first in-flight row
+        float *e_all = nullptr, *s_all = nullptr;
+        int rc = RD_OK;
+        if (n > 0) {
+            RD_TRY(s->mem.get(&e_all, (size_t)n * h * sizeof(float)));
+            rc = s->mem.get(&s_all, (size_t)n * h * sizeof(float));
+        }
+        for (int pass = 0; pass < r + 2 && !rc && n > 0; pass++) {
+            // pass 0: P and s_0 for every chunk; passes 1..r: one simultaneous application of R;
+            // pass r+1: coda layers (fills the coda cache; no head).
+            for (int c0 = 0; c0 < n && !rc; c0 += s->R) {
+                const int nr = std::min(s->R, n - c0);
+                fill_rows_kernel<<<(s->R + 127) / 128, 128, 0, s->stream>>>(seq, c0, nr, s->R, s->row_pos, s->row_seq);
+                s->stats.kernel_launches++;
+                float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
+                float* zc = s_all + (size_t)c0 * h;
+                if (pass == 0) {
+                    rc = prelude(s, nr);
+                    if (rc) break;
+                    cudaMemcpyAsync(ec, s->x, (size_t)nr * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream);
+                    init_state_kernel<<<nr, 128, 0, s->stream>>>(s->row_pos, s->row_seq, s->row_steps, 0, h,
+                                                                 c.init_sigma, s->sc.seed, zc, h);
+                    s->stats.kernel_launches++;
+                } else if (pass <= r) {
+                    rc = core(s, ec, zc, zc, nr);
+                } else {
+                    rc = coda(s, zc, nr, false);
+                }
+            }
+        }
+        if (!rc) {
+            cudaError_t e = cudaStreamSynchronize(s->stream);
+            if (e == cudaSuccess) e = cudaGetLastError();
+            if (e != cudaSuccess) rc = cuda_fail(e, "prefill", __LINE__);
+        }
+        if (e_all) s->mem.release(e_all);
+        if (s_all) s->mem.release(s_all);
+        if (rc) return rc;
+        // sequence state: |y_frozen| = L, one fresh in-flight row at position L-1
+        const int one = 1, zero = 0, isdone = s->sc.max_new_tokens <= 0 ? 1 : 0;
+        const int slot = seq * s->sc.max_window + (L - 1) % s->sc.max_window;
+        CU(cudaMemcpy(s->n_prompt + seq, &L, sizeof(int), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(s->n_committed + seq, &L, sizeof(int), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(s->win_len + seq, isdone ? &zero : &one, sizeof(int), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(s->done + seq, &isdone, sizeof(int), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(s->row_steps + slot, &zero, sizeof(int), cudaMemcpyHostToDevice));
+        CU(cudaMemcpy(s->row_iters + slot, &zero, sizeof(int), cudaMemcpyHostToDevice));
+        return RD_OK;
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// C ABI: steps and inspection
+// ---------------------------------------------------------------------------------------------
+static bool any_prefilled(const rd_session* s) {
+    for (char c : s->prefilled) if (c) return true;
+    return false;
+}
+
+extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r) {
+    if (!s || !prompt || seq < 0 || seq >= s->sc.batch || n_prompt < 1 || r < 0) return RD_E_INVALID_ARG;
+    if ((long long)n_prompt + s->sc.max_new_tokens > s->sc.max_context) return RD_E_CAPACITY;
+    for (int i = 0; i < n_prompt; i++)
+        if (prompt[i] < 0 || prompt[i] >= s->m->cfg.vocab) return RD_E_INVALID_ARG;
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::prefill(s, seq, prompt, n_prompt, r)
+                                              : Eng<float>::prefill(s, seq, prompt, n_prompt, r);
+    if (rc == RD_OK) { s->prefilled[seq] = 1; s->wave_open[seq] = 0; }
+    return rc;
+}
+
+extern "C" int rd_ar_step(rd_session* s, int32_t r) {
+    if (!s || r < 1) return RD_E_INVALID_ARG;
+    if (!any_prefilled(s)) return RD_E_STATE;
+    for (int b = 0; b < s->sc.batch; b++)
+        if (s->prefilled[b] && s->wave_open[b]) return RD_E_STATE;
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, 1, r, 0.f) : Eng<float>::decode_step(s, 1, r, 0.f);
+    if (rc == RD_OK) s->stats.ar_steps++;
+    return rc;
+}
+
+extern "C" int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, float exit_threshold) {
+    if (!s || window < 1 || inner_iters < 1 || exit_threshold != exit_threshold) return RD_E_INVALID_ARG;
+    if (window > s->sc.max_window) return RD_E_CAPACITY;
+    if (!any_prefilled(s)) return RD_E_STATE;
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, window, inner_iters, exit_threshold)
+                                              : Eng<float>::decode_step(s, window, inner_iters, exit_threshold);
+    if (rc == RD_OK) {
+        s->stats.df_steps++;
+        if (window > 1)
+            for (int b = 0; b < s->sc.batch; b++) if (s->prefilled[b]) s->wave_open[b] = 1;
+    }
+    return rc;
+}
+
+extern "C" int rd_sync(rd_session* s) {
+    if (!s) return RD_E_INVALID_ARG;
+    CU(cudaStreamSynchronize(s->stream));
+    int st[4] = {0, 0, 0, 0};
+    CU(cudaMemcpy(st, s->status, sizeof st, cudaMemcpyDeviceToHost));
+    return st[0] ? RD_E_TIMEOUT : RD_OK;
+}
+
+extern "C" int rd_committed(rd_session* s, int32_t seq, int32_t* n_tokens, int32_t* done) {
+    if (!s || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    RD_TRY(rd_sync(s));
+    int n = 0, d = 0;
+    CU(cudaMemcpy(&n, s->n_committed + seq, sizeof(int), cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(&d, s->done + seq, sizeof(int), cudaMemcpyDeviceToHost));
+    if (n_tokens) *n_tokens = n;
+    if (done) *done = s->prefilled[seq] ? d : 0;
+    return RD_OK;
+}
+
+extern "C" int rd_get_tokens(rd_session* s, int32_t seq, int32_t* dst, int32_t cap, int32_t* n_written) {
+    if (!s || !dst || cap < 0 || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    int n = 0;
+    RD_TRY(rd_committed(s, seq, &n, nullptr));
+    n = std::min(n, cap);
+    if (n > 0) CU(cudaMemcpy(dst, s->tokens + (size_t)seq * s->tok_stride, (size_t)n * sizeof(int), cudaMemcpyDeviceToHost));
+    if (n_written) *n_written = n;
+    return RD_OK;
+}
+
+extern "C" int rd_last_step_rows(rd_session* s, int32_t seq, int32_t* first_pos, int32_t* n_rows) {
+    if (!s || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    if (s->stats.df_steps + s->stats.ar_steps == 0) return RD_E_STATE;
+    RD_TRY(rd_sync(s));
+    int f = 0, n = 0;
+    CU(cudaMemcpy(&f, s->step_first + seq, sizeof(int), cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(&n, s->step_n + seq, sizeof(int), cudaMemcpyDeviceToHost));
+    if (first_pos) *first_pos = f;
+    if (n_rows) *n_rows = n;
+    return RD_OK;
+}
+
+extern "C" int rd_debug_read(rd_session* s, int32_t what, int32_t seq, void* dst, size_t bytes) {
+    if (!s || !dst) return RD_E_INVALID_ARG;
+    int f = 0, n = 0;
+    RD_TRY(rd_last_step_rows(s, seq, &f, &n));
+    const rd_config& c = s->m->cfg;
+    size_t row_bytes = 0;
+    const char* base = nullptr;
+    switch (what) {
+        case RD_DBG_LATENTS: row_bytes = (size_t)c.hidden * 4; base = (const char*)s->z; break;
+        case RD_DBG_EMBED: row_bytes = (size_t)c.hidden * 4; base = (const char*)s->e; break;
+        case RD_DBG_DELTA: row_bytes = 4; base = (const char*)s->delta; break;
+        case RD_DBG_DRAFTS: row_bytes = 4; base = (const char*)s->draft; break;
+        case RD_DBG_LOGITS:
+            if (!s->sc.keep_logits) return RD_E_STATE;
+            row_bytes = (size_t)c.vocab * 4; base = (const char*)s->logits; break;
+        default: return RD_E_INVALID_ARG;
+    }
+    if (bytes < row_bytes * n) return RD_E_INVALID_ARG;
+    for (int i = 0; i < n; i++) {
+        const int slot = seq * s->sc.max_window + (f + i) % s->sc.max_window;
+        CU(cudaMemcpy((char*)dst + (size_t)i * row_bytes, base + (size_t)slot * row_bytes, row_bytes, cudaMemcpyDeviceToHost));
+    }
+    return RD_OK;
+}
+
+extern "C" int rd_debug_force_tokens(rd_session* s, int32_t seq, int32_t first_pos, const int32_t* tokens, int32_t n) {
+    if (!s || !tokens || seq < 0 || seq >= s->sc.batch || n < 0 || !s->prefilled[seq]) return RD_E_INVALID_ARG;
+    RD_TRY(rd_sync(s));
+    int np = 0;
+    CU(cudaMemcpy(&np, s->n_prompt + seq, sizeof(int), cudaMemcpyDeviceToHost));
+    if (first_pos < np || (long long)first_pos + n > s->tok_stride) return RD_E_INVALID_ARG;
+    for (int i = 0; i < n; i++)
+        if (tokens[i] < 0 || tokens[i] >= s->m->cfg.vocab) return RD_E_INVALID_ARG;
+    if (n) CU(cudaMemcpy(s->tokens + (size_t)seq * s->tok_stride + first_pos, tokens, (size_t)n * sizeof(int), cudaMemcpyHostToDevice));
+    return RD_OK;
+}
+
+extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq, int32_t pos0,
+                                int32_t n, float* dst) {
+    if (!s || !dst || block < 0 || block > 2 || (which != 0 && which != 1) || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    const rd_config& c = s->m->cfg;
+    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 + n > s->sc.max_context) return RD_E_INVALID_ARG;
+    RD_TRY(rd_sync(s));
+    if (n == 0) return RD_OK;
+    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride + (size_t)pos0 * c.hidden;
+    const size_t cnt = (size_t)n * c.hidden;
+    const char* src = (const char*)(which ? s->Vc[block] : s->Kc[block]) + off * s->m->esz;
+    if (c.dtype == RD_F32) {
+        CU(cudaMemcpy(dst, src, cnt * 4, cudaMemcpyDeviceToHost));
+        return RD_OK;
+    }
+    float* tmp = nullptr;
+    CU(cudaMalloc((void**)&tmp, cnt * 4));
+    widen_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, tmp, cnt);
+    cudaError_t e = cudaStreamSynchronize(s->stream);
+    if (e == cudaSuccess) e = cudaMemcpy(dst, tmp, cnt * 4, cudaMemcpyDeviceToHost);
+    cudaFree(tmp);
+    if (e != cudaSuccess) return cuda_fail(e, "read_kv", __LINE__);
+    return RD_OK;
+}
+
+extern "C" int rd_stats(rd_session* s, rd_stats_t* out) {
+    if (!s || !out) return RD_E_INVALID_ARG;
+    RD_TRY(rd_sync(s));
+    unsigned long long cnt[8];
+    CU(cudaMemcpy(cnt, s->counters, sizeof cnt, cudaMemcpyDeviceToHost));
+    *out = s->stats;
+    out->rows_prelude = cnt[0];
+    out->rows_core = cnt[1];
+    out->rows_coda = cnt[2];
+    out->tokens_committed = cnt[3];
+    return RD_OK;
+}

@@ -1,0 +1,104 @@
+"""Lock-step comparison of the CUDA library (through the C ABI) with the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+import paper_2510_14961_b200 as rd
+import rd_inputs
+from oracle import rd_oracle as orc
+
+
+def gpu_model(shape, weights, bf16=False, **kw):
+    specs = rd_inputs.tensor_specs(**rd_inputs.shape_args(shape), tie_embeddings=kw.get("tie_embeddings", True))
+    tensors = [np.ascontiguousarray(weights[name], dtype=np.float32) for name, _, _ in specs]
+    return rd.Model(shape["hidden"], shape["n_heads"], shape["head_dim"], shape["mlp_inner"], shape["n_prelude"],
+                    shape["n_core"], shape["n_coda"], shape["vocab"], tensors,
+                    dtype=rd.RD_BF16 if bf16 else rd.RD_F32, **kw)
+
+
+class Tolerance:
+    def __init__(self, abs_tol, rel_tol=0.0):
+        self.abs_tol, self.rel_tol = abs_tol, rel_tol
+
+    def excess(self, got, want):
+        """max over elements of |got-want| - (abs + rel*|want|); <= 0 means within tolerance."""
+        return float(np.max(np.abs(got - want) - (self.abs_tol + self.rel_tol * np.abs(want))))
+
+
+class LockStep:
+    """Runs the oracle sampler and a GPU session side by side on one or more sequences and compares
+    every step: rows processed, latents, logits, delta, drafts, commit counts.
+
+    A draft mismatch is admissible only when the oracle's own top-2 gap (of the scores that decide
+    the token) is below `tie_gap`; the oracle then follows the GPU's token so that both continue
+    from the same y_current.  The fp32 configuration uses tie_gap = 0: any mismatch fails."""
+
+    def __init__(self, sampler: orc.Sampler, session: rd.Session, seqs, tol: Tolerance, tie_gap=0.0,
+                 check_logits=True):
+        self.sm, self.sess, self.seqs, self.tol, self.tie_gap = sampler, session, seqs, tol, tie_gap
+        self.check_logits = check_logits
+        self.near_ties = 0
+        self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0}
+        self.steps = 0
+
+    def _scores(self, logits, sq, token_pos):
+        l32 = logits.astype(np.float32)
+        if self.sm.temperature <= 0:
+            return l32
+        return l32 / np.float32(self.sm.temperature) + orc.gumbel_noise(self.sm.seed, sq.seq_id, token_pos,
+                                                                        l32.shape[0])
+
+    def compare(self, infos, delta_checked=True):
+        self.steps += 1
+        for sq, info in zip(self.seqs, infos):
+            b = sq.seq_id
+            if info is None:
+                continue
+            f, n = self.sess.last_step_rows(b)
+            assert n == len(info["pos"]) and (n == 0 or f == int(info["pos"][0])), \
+                f"step {self.steps} seq {b}: GPU rows ({f},{n}) vs oracle {info['pos']}"
+            z = self.sess.debug_read(rd.RD_DBG_LATENTS, b)
+            ex = self.tol.excess(z, info["z"])
+            self.max_err["z"] = max(self.max_err["z"], float(np.abs(z - info["z"]).max()))
+            assert ex <= 0, f"step {self.steps} seq {b}: latents off by {np.abs(z - info['z']).max():.3e}"
+            if self.check_logits:
+                lg = self.sess.debug_read(rd.RD_DBG_LOGITS, b)
+                self.max_err["logits"] = max(self.max_err["logits"], float(np.abs(lg - info["logits"]).max()))
+                assert self.tol.excess(lg, info["logits"]) <= 0, \
+                    f"step {self.steps} seq {b}: logits off by {np.abs(lg - info['logits']).max():.3e}"
+            if delta_checked and "delta" in info:
+                dl = self.sess.debug_read(rd.RD_DBG_DELTA, b)
+                fin = np.isfinite(info["delta"])
+                if fin.any():
+                    self.max_err["delta"] = max(self.max_err["delta"], float(np.abs(dl - info["delta"])[fin].max()))
+            drafts = self.sess.debug_read(rd.RD_DBG_DRAFTS, b)
+            for i in range(n):
+                if drafts[i] == info["drafts"][i]:
+                    continue
+                sc = self._scores(info["logits"][i], sq, int(info["pos"][i]) + 1)
+                gap = float(sc[info["drafts"][i]] - sc[drafts[i]])
+                assert 0 <= gap <= self.tie_gap, \
+                    f"step {self.steps} seq {b} row {i}: GPU token {drafts[i]} vs oracle {info['drafts'][i]}, gap {gap:.3e}"
+                self.near_ties += 1
+                self.sm.force_draft(sq, int(info["pos"][i]) + 1, int(drafts[i]))
+            ncom, done = self.sess.committed(b)
+            assert ncom == sq.n_committed and done == sq.done, \
+                f"step {self.steps} seq {b}: committed {ncom}/{done} vs oracle {sq.n_committed}/{sq.done}"
+
+    def df(self, window, inner, eps):
+        infos = [self.sm.df_step(sq, window, inner, eps) for sq in self.seqs]
+        self.sess.df_step(window, inner, eps)
+        self.compare(infos)
+
+    def ar(self, r):
+        infos = [self.sm.ar_step(sq, r) for sq in self.seqs]
+        self.sess.ar_step(r)
+        self.compare(infos, delta_checked=False)
+
+    def all_done(self):
+        return all(sq.done for sq in self.seqs)
+
+    def final_tokens_equal(self):
+        for sq in self.seqs:
+            got = self.sess.tokens(sq.seq_id)
+            assert np.array_equal(got, sq.committed()), f"seq {sq.seq_id}: final tokens differ"
