@@ -165,6 +165,19 @@ int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which,
 /* rd_stats -- counters since session creation (host pointer out). */
 int rd_stats(rd_session* s, rd_stats_t* out);
 
+/* rd_profile_enable / rd_profile_read -- measurement aid.  While enabled, every GEMM launch and
+ * every attention launch is bracketed by a pair of CUDA events recorded on the session's stream;
+ * rd_profile_read synchronises, sums the elapsed times of the pairs recorded since the last read
+ * and resets the list.  Bytes are the algorithmic ones: weight bytes of each GEMM (n_out * K *
+ * element size), and for attention the K and V rows each (sequence, layer) must read once.
+ * At most 16384 pairs are kept between reads; later launches are then not bracketed. */
+typedef struct {
+    uint64_t gemm_launches;  double gemm_ms;  uint64_t gemm_weight_bytes;
+    uint64_t attn_launches;  double attn_ms;  uint64_t attn_kv_bytes;
+} rd_profile_t;
+int rd_profile_enable(rd_session* s, int32_t on);
+int rd_profile_read(rd_session* s, rd_profile_t* out);
+
 /* rd_set_gemm_path -- 0: SIMT kernels everywhere; 1 (default for RD_BF16): tcgen05 tensor-core
  * GEMMs where the shape allows.  For measurement and parity tests. */
 int rd_set_gemm_path(rd_session* s, int32_t path);

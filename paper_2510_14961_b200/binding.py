@@ -17,7 +17,7 @@ RD_DBG_LATENTS, RD_DBG_DELTA, RD_DBG_DRAFTS, RD_DBG_LOGITS, RD_DBG_EMBED = 0, 1,
 EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_prefill", "rd_ar_step",
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
-           "rd_last_cuda_error"]
+           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read"]
 
 
 class RdConfig(C.Structure):
@@ -35,6 +35,11 @@ class RdSessionConfig(C.Structure):
 class RdStats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("df_steps", "ar_steps", "rows_prelude", "rows_core", "rows_coda",
                                           "tokens_committed", "kernel_launches", "tc_gemm_launches")]
+
+
+class RdProfile(C.Structure):
+    _fields_ = [("gemm_launches", C.c_uint64), ("gemm_ms", C.c_double), ("gemm_weight_bytes", C.c_uint64),
+                ("attn_launches", C.c_uint64), ("attn_ms", C.c_double), ("attn_kv_bytes", C.c_uint64)]
 
 
 class RdError(RuntimeError):
@@ -72,6 +77,8 @@ def lib():
         L.rd_debug_read_kv.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
         L.rd_stats.argtypes = [vp, C.POINTER(RdStats)]
         L.rd_set_gemm_path.argtypes = [vp, i32]
+        L.rd_profile_enable.argtypes = [vp, i32]
+        L.rd_profile_read.argtypes = [vp, C.POINTER(RdProfile)]
         L.rd_strerror.argtypes = [C.c_int]
         L.rd_strerror.restype = C.c_char_p
         L.rd_last_cuda_error.restype = C.c_char_p
@@ -206,3 +213,11 @@ class Session:
 
     def set_gemm_path(self, path):
         _check(lib().rd_set_gemm_path(self.handle, path), "rd_set_gemm_path")
+
+    def profile_enable(self, on=True):
+        _check(lib().rd_profile_enable(self.handle, 1 if on else 0), "rd_profile_enable")
+
+    def profile_read(self):
+        pr = RdProfile()
+        _check(lib().rd_profile_read(self.handle, C.byref(pr)), "rd_profile_read")
+        return {k: getattr(pr, k) for k, _ in RdProfile._fields_}

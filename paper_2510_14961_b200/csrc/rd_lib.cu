@@ -236,9 +236,37 @@ struct rd_session {
     TcAct t_act_h, t_act_2h, t_act_i;
     // host state
     std::vector<char> prefilled, wave_open;
+    std::vector<int> host_prompt_len, host_steps;   // host-side view, for byte accounting only
     int gemm_path = 0;
     rd_stats_t stats;
+    // measurement aid: event pairs around GEMM (kind 0) and attention (kind 1) launches
+    struct Bracket { cudaEvent_t a, b; int kind; uint64_t bytes; };
+    bool profiling = false;
+    std::vector<Bracket> brackets;
+    std::vector<cudaEvent_t> event_pool;
+    uint64_t ctx_total = 0;   // host-side upper bound of sum over sequences of context length
+    ~rd_session() {
+        for (Bracket& b : brackets) { cudaEventDestroy(b.a); cudaEventDestroy(b.b); }
+        for (cudaEvent_t e : event_pool) cudaEventDestroy(e);
+    }
 };
+
+// RAII-free helpers: open a bracket before a launch, close it after.
+static int bracket_open(rd_session* s, int kind, uint64_t bytes) {
+    if (!s->profiling || s->brackets.size() >= 16384) return -1;
+    rd_session::Bracket b;
+    b.kind = kind; b.bytes = bytes;
+    for (cudaEvent_t* e : {&b.a, &b.b}) {
+        if (!s->event_pool.empty()) { *e = s->event_pool.back(); s->event_pool.pop_back(); }
+        else if (cudaEventCreate(e) != cudaSuccess) return -1;
+    }
+    cudaEventRecord(b.a, s->stream);
+    s->brackets.push_back(b);
+    return (int)s->brackets.size() - 1;
+}
+static void bracket_close(rd_session* s, int idx) {
+    if (idx >= 0) cudaEventRecord(s->brackets[idx].b, s->stream);
+}
 
 #define LAUNCHED(s)                  \
     do {                             \
@@ -330,6 +358,8 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     if (rc) { delete s; return rc; }
     s->prefilled.assign(B, 0);
     s->wave_open.assign(B, 0);
+    s->host_prompt_len.assign(B, 0);
+    s->host_steps.assign(B, 0);
     *out = s;
     return RD_OK;
 }
@@ -353,10 +383,11 @@ template <typename T> struct Eng {
     // the tensor-core path (bf16 only).
     static int gemm(rd_session* s, const T* A, size_t lda, const TcAct* ta, const T* W, const TcWeight* tw, int K,
                     int n_out, float* Y, size_t ldy, const float* resid, int n_rows) {
+        const int br = bracket_open(s, 0, (uint64_t)n_out * K * sizeof(T));
         if (sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid) {
             const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, Y, ldy, resid, n_rows, s->partial,
                                    s->partial_elems, s->status, &s->stats.kernel_launches);
-            if (rc == RD_OK) { s->stats.tc_gemm_launches++; return RD_OK; }
+            if (rc == RD_OK) { s->stats.tc_gemm_launches++; bracket_close(s, br); return RD_OK; }
             if (rc != RD_E_INVALID_ARG) return rc;   // INVALID_ARG: shape not taken, fall through
         }
         const int warps = 8;
@@ -370,6 +401,7 @@ template <typename T> struct Eng {
             gemm_simt_kernel<T, 8><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
         }
         LAUNCHED(s);
+        bracket_close(s, br);
         return RD_OK;
     }
 
@@ -387,10 +419,12 @@ template <typename T> struct Eng {
         rope_kv_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->qkv, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h,
                                                           c.head_dim, (T*)s->q_t, Kc, Vc, s->seq_stride);
         LAUNCHED(s);
+        const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         attn_row_kernel<T><<<dim3(n_rows, c.n_heads), 128, 0, s->stream>>>(
             (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc, s->seq_stride, h, c.head_dim,
             (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
         LAUNCHED(s);
+        bracket_close(s, br);
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, x, h, x, n_rows));
         rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g2, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
         LAUNCHED(s);
@@ -447,6 +481,13 @@ template <typename T> struct Eng {
     static int decode_step(rd_session* s, int window, int inner, float eps) {
         const rd_config& c = s->m->cfg;
         const int n = s->n_slots, h = c.hidden, B = s->sc.batch;
+        // the leading edge of a wavefront advances by at most one position per step
+        s->ctx_total = 0;
+        for (int b = 0; b < B; b++)
+            if (s->prefilled[b]) {
+                s->host_steps[b]++;
+                s->ctx_total += std::min(s->host_prompt_len[b] + s->host_steps[b], s->host_prompt_len[b] + s->sc.max_new_tokens);
+            }
         plan_rows_kernel<<<(n + 127) / 128, 128, 0, s->stream>>>(s->n_committed, s->win_len, s->done, B,
                                                                  s->sc.max_window, s->row_pos, s->row_seq,
                                                                  s->step_first, s->step_n);
@@ -539,7 +580,10 @@ extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int
         if (prompt[i] < 0 || prompt[i] >= s->m->cfg.vocab) return RD_E_INVALID_ARG;
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::prefill(s, seq, prompt, n_prompt, r)
                                               : Eng<float>::prefill(s, seq, prompt, n_prompt, r);
-    if (rc == RD_OK) { s->prefilled[seq] = 1; s->wave_open[seq] = 0; }
+    if (rc == RD_OK) {
+        s->prefilled[seq] = 1; s->wave_open[seq] = 0;
+        s->host_prompt_len[seq] = n_prompt; s->host_steps[seq] = 0;
+    }
     return rc;
 }
 
@@ -679,5 +723,28 @@ extern "C" int rd_stats(rd_session* s, rd_stats_t* out) {
     out->rows_core = cnt[1];
     out->rows_coda = cnt[2];
     out->tokens_committed = cnt[3];
+    return RD_OK;
+}
+
+extern "C" int rd_profile_enable(rd_session* s, int32_t on) {
+    if (!s) return RD_E_INVALID_ARG;
+    s->profiling = on != 0;
+    return RD_OK;
+}
+
+extern "C" int rd_profile_read(rd_session* s, rd_profile_t* out) {
+    if (!s || !out) return RD_E_INVALID_ARG;
+    RD_TRY(rd_sync(s));
+    memset(out, 0, sizeof *out);
+    for (rd_session::Bracket& b : s->brackets) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, b.a, b.b) == cudaSuccess) {
+            if (b.kind == 0) { out->gemm_launches++; out->gemm_ms += ms; out->gemm_weight_bytes += b.bytes; }
+            else { out->attn_launches++; out->attn_ms += ms; out->attn_kv_bytes += b.bytes; }
+        }
+        s->event_pool.push_back(b.a);
+        s->event_pool.push_back(b.b);
+    }
+    s->brackets.clear();
     return RD_OK;
 }

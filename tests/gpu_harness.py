@@ -38,6 +38,7 @@ class LockStep:
         self.sm, self.sess, self.seqs, self.tol, self.tie_gap = sampler, session, seqs, tol, tie_gap
         self.check_logits = check_logits
         self.near_ties = 0
+        self.n_drafts = 0
         self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0}
         self.steps = 0
 
@@ -72,6 +73,7 @@ class LockStep:
                 if fin.any():
                     self.max_err["delta"] = max(self.max_err["delta"], float(np.abs(dl - info["delta"])[fin].max()))
             drafts = self.sess.debug_read(rd.RD_DBG_DRAFTS, b)
+            self.n_drafts += n
             for i in range(n):
                 if drafts[i] == info["drafts"][i]:
                     continue

@@ -1,0 +1,121 @@
+"""GPU parity, bf16 configurations: reduced-width twin of the 3.5B shape (head_dim 96, 2/4/2 layers)
+in lock step with the oracle's bf16-contract mode, and truncated runs at the full 3.5B shape.
+Tolerance (stated by the benchmark spec): |err| <= 5e-2 + 2e-2 |want| on latents and logits; tokens identical
+except at near-ties of the deciding scores, which are counted and bounded."""
+import numpy as np
+import pytest
+
+import paper_2510_14961_b200 as rd
+import rd_inputs
+from oracle import rd_oracle as orc
+from gpu_harness import LockStep, Tolerance, gpu_model
+from helpers import make_oracle
+
+pytestmark = pytest.mark.gpu
+TOL = Tolerance(5e-2, 2e-2)
+# Two bf16 pipelines that sum in different orders round differently at every bf16 store; the
+# resulting noise floor on logits is ~1.5e-2 here (inside the stated tolerance).  A GPU/oracle token
+# mismatch is admissible only if the oracle's own score gap between the two tokens is below
+# TIE_GAP; top-2 gaps average ~0.3, so a few percent of the arg-max decisions are such near-ties.
+TIE_GAP = 3e-2
+MAX_TIE_FRACTION = 0.08
+
+
+def _ties_ok(ls):
+    return ls.near_ties <= max(2, int(MAX_TIE_FRACTION * ls.n_drafts))
+
+
+def _setup(shape, W, max_new, batch=1, temperature=0.0, cap=64, max_ctx=256, seed=0, gemm_path=None,
+           dtype=np.float64, std=0.02, **wkw):
+    model, w = make_oracle(shape, seed=seed, std=std, gain_jitter=0.0, bf16=True, contract=True, max_ctx=max_ctx,
+                           dtype=dtype, **wkw)
+    gm = gpu_model(shape, w, bf16=True)
+    sess = rd.Session(gm, batch=batch, max_context=max_ctx, max_window=W, max_iters_per_pos=cap,
+                      max_new_tokens=max_new, keep_logits=True, temperature=temperature, seed=seed + 7)
+    if gemm_path is not None:
+        sess.set_gemm_path(gemm_path)      # raises if the tensor-core path is unavailable
+    sm = orc.Sampler(model, seed=seed + 7, temperature=temperature, max_iters_per_pos=cap)
+    return model, gm, sess, sm
+
+
+def _prefill_both(sm, sess, shape, lens, r, max_new, seed=0):
+    seqs = []
+    for b, L in enumerate(lens):
+        prompt = rd_inputs.make_prompt(int(L), shape["vocab"], seed=seed + b)
+        seqs.append(sm.prefill(b, prompt, r, max_new))
+        sess.prefill(b, prompt, r)
+    return seqs
+
+
+def _run(ls, W, inner, eps, max_steps=2000):
+    for _ in range(max_steps):
+        if ls.all_done():
+            break
+        ls.df(W, inner, eps)
+    assert ls.all_done()
+    ls.final_tokens_equal()
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("W,inner,eps,temperature", [(4, 1, 0.0, 0.0), (16, 2, 0.0, 0.0), (8, 1, 1e-3, 0.0),
+                                                     (16, 1, 1e-3, 1.0)])
+def test_twin_df_modes(path, W, inner, eps, temperature):
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, W, 24, temperature=temperature, cap=16, gemm_path=path)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [40], 4, 24)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    _run(ls, W, inner, eps)
+    print(f"path {path} W {W}: steps {ls.steps}, near-ties {ls.near_ties}, max err {ls.max_err}")
+    assert _ties_ok(ls)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_twin_ar_and_window1_identity(path):
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 1, 8, gemm_path=path)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [20], 4, 8)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    while not ls.all_done():
+        ls.ar(6)
+    ls.final_tokens_equal()
+    ar_tokens, ar_z = sess.tokens(0).copy(), sess.debug_read(rd.RD_DBG_LATENTS, 0).copy()
+    sess2 = rd.Session(gm, batch=1, max_context=256, max_window=1, max_new_tokens=8, keep_logits=True, seed=7)
+    sess2.set_gemm_path(path)
+    sess2.prefill(0, rd_inputs.make_prompt(20, 4096, seed=0), 4)
+    for _ in range(8):
+        sess2.df_step(1, 6, 0.0)
+    assert np.array_equal(sess2.tokens(0), ar_tokens)
+    assert np.array_equal(sess2.debug_read(rd.RD_DBG_LATENTS, 0), ar_z)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_twin_batched_ragged_sampling(path):
+    """Batched serving shape: ragged prompts, temperature sampling on the shared counter stream,
+    adaptive exit."""
+    lens = rd_inputs.make_prompt_lengths(4, 3, 60, seed=3)
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 8, 16, batch=4, temperature=1.0, cap=12, gemm_path=path)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 3, 16)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    _run(ls, 8, 1, 1e-3)
+    assert _ties_ok(ls)
+
+
+def test_twin_long_prefix_attention():
+    """A prompt spanning many attention tiles (long-context shape, reduced width)."""
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 8, 10, max_ctx=1200)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [1100], 1, 10)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    _run(ls, 8, 1, 0.0)
+    assert _ties_ok(ls)
+
+
+def test_gpu_run_to_run_bit_identical():
+    """Fixed-order reductions everywhere: two runs give the same bits."""
+    outs = []
+    for _ in range(2):
+        model, gm, sess, sm = _setup(rd_inputs.TWIN, 8, 12)
+        sess.prefill(0, rd_inputs.make_prompt(30, 4096, seed=1), 3)
+        for _ in range(19):
+            sess.df_step(8, 1, 0.0)
+        outs.append((sess.tokens(0).copy(), sess.debug_read(rd.RD_DBG_LATENTS, 0).copy(),
+                     sess.debug_read(rd.RD_DBG_LOGITS, 0).copy()))
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
