@@ -319,9 +319,11 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if ((rc = s->mem.get(&s->z_prev, R * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->logits, (size_t)s->n_slots * V * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->delta, R * sizeof(float)))) break;
-        if ((rc = s->mem.get(&s->act_h, R * h * es))) break;
-        if ((rc = s->mem.get(&s->act_2h, R * 2 * h * es))) break;
-        if ((rc = s->mem.get(&s->act_i, R * I * es))) break;
+        // GEMM-input buffers hold at least 256 rows so that the widest TMA row box stays inside
+        const size_t Ra = std::max<size_t>(R, 256);
+        if ((rc = s->mem.get(&s->act_h, Ra * h * es))) break;
+        if ((rc = s->mem.get(&s->act_2h, Ra * 2 * h * es))) break;
+        if ((rc = s->mem.get(&s->act_i, Ra * I * es))) break;
         if ((rc = s->mem.get(&s->q_t, R * h * es))) break;
         for (int blk = 0; blk < 3 && !rc; blk++) {
             const size_t n = (size_t)n_layers_of(c, blk) * B * s->seq_stride * es;
@@ -349,9 +351,9 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if (m->tc_ok) {
             s->partial_elems = tc_partial_elems(R, c);
             if ((rc = s->mem.get(&s->partial, s->partial_elems * sizeof(float)))) break;
-            bool ok = tc_make_act(&s->t_act_h, s->act_h, s->R, c.hidden) == RD_OK;
-            ok &= tc_make_act(&s->t_act_2h, s->act_2h, s->R, 2 * c.hidden) == RD_OK;
-            ok &= tc_make_act(&s->t_act_i, s->act_i, s->R, c.mlp_inner) == RD_OK;
+            bool ok = tc_make_act(&s->t_act_h, s->act_h, (int)Ra, c.hidden) == RD_OK;
+            ok &= tc_make_act(&s->t_act_2h, s->act_2h, (int)Ra, 2 * c.hidden) == RD_OK;
+            ok &= tc_make_act(&s->t_act_i, s->act_i, (int)Ra, c.mlp_inner) == RD_OK;
             s->gemm_path = ok ? 1 : 0;
         }
     } while (0);

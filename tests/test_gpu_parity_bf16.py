@@ -66,6 +66,7 @@ def test_twin_df_modes(path, W, inner, eps, temperature):
     _run(ls, W, inner, eps)
     print(f"path {path} W {W}: steps {ls.steps}, near-ties {ls.near_ties}, max err {ls.max_err}")
     assert _ties_ok(ls)
+    assert (sess.stats()["tc_gemm_launches"] > 0) == (path == 1)
 
 
 @pytest.mark.parametrize("path", [0, 1])
