@@ -1,0 +1,240 @@
+// Windowed flash-decode attention for the bf16 path.
+//
+// One CTA takes one (query group, head, KV split).  A query group is a set of up to 64 rows of ONE
+// sequence (the in-flight wavefront of a sequence during decode, 64 consecutive prompt positions
+// during prefill).  The row at position p attends cache entries 0..p of its sequence: committed
+// prefix and the in-flight rows <= p as overwritten this pass (shared KV cache, Section 3.2;
+// causal, left to right only).  K and V tiles of 64 keys stream through shared memory once per CTA
+// (16-byte cp.async, double buffered) and are reused by every query of the group, so the KV
+// prefix is read once per (sequence, head) for the whole wavefront.  Each warp owns 16 queries:
+// S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with an online
+// softmax in fp32; P is rounded to bf16 for the second product.  Splits write (m, l, O) partials
+// that a second kernel merges in split order (deterministic).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace rd {
+
+constexpr int ATT_KT = 64;          // keys per tile
+constexpr int ATT_QMAX = 64;        // queries per group
+constexpr int ATT_MAX_SPLITS = 16;
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+    const int sz = valid ? 16 : 0;                      // 0 bytes read => 16 bytes of zeros written
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t* r, const void* p) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t* r, const void* p) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int D> struct AttCfg {
+    static constexpr int LD = D + 8;    // padded row (elements): ldmatrix rows fall in distinct banks
+    static constexpr int SMEM = (ATT_QMAX * LD + 4 * ATT_KT * LD) * 2 + ATT_QMAX * 4;
+};
+
+// part_o: [row][head][split][D] unnormalised outputs; part_ml: [row][head][split][2] = (max, sum),
+// the max in the log2 domain of the scaled scores.
+template <int D>
+__global__ void __launch_bounds__(128)
+attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
+                   const int* __restrict__ row_seq, int rows_per_group, int n_rows,
+                   const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
+                   int hidden, float scale_log2, int n_splits, float* __restrict__ part_o,
+                   float* __restrict__ part_ml) {
+    constexpr int LD = AttCfg<D>::LD;
+    constexpr int CH = D / 8;           // 16-byte chunks per row
+    extern __shared__ __align__(16) uint8_t att_smem[];
+    __nv_bfloat16* Qs = (__nv_bfloat16*)att_smem;
+    __nv_bfloat16* Ks = Qs + ATT_QMAX * LD;               // [2][KT][LD]
+    __nv_bfloat16* Vs = Ks + 2 * ATT_KT * LD;             // [2][KT][LD]
+    int* pos_s = (int*)(Vs + 2 * ATT_KT * LD);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int hd = blockIdx.x, H = gridDim.x, sp = blockIdx.z;
+    const int r0 = blockIdx.y * rows_per_group;
+    const int nq = min(rows_per_group, n_rows - r0);
+    if (tid < ATT_QMAX) pos_s[tid] = tid < nq ? row_pos[r0 + tid] : -1;
+    __syncthreads();
+    int kv_len = 0;
+    for (int i = 0; i < ATT_QMAX; i++) kv_len = max(kv_len, pos_s[i] + 1);
+    const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
+    const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
+    const int seq = row_seq[r0];
+    const __nv_bfloat16* kbase = Kc + (size_t)seq * seq_stride + (size_t)hd * D;
+    const __nv_bfloat16* vbase = Vc + (size_t)seq * seq_stride + (size_t)hd * D;
+
+    for (int c = tid; c < ATT_QMAX * CH; c += 128) {
+        const int r = c / CH, ch = c % CH;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)(r0 + r) * hidden + hd * D + ch * 8);
+        *reinterpret_cast<uint4*>(Qs + r * LD + ch * 8) = v;
+    }
+    auto load_tile = [&](int t, int buf) {
+        const int key0 = t * ATT_KT;
+        for (int c = tid; c < ATT_KT * CH; c += 128) {
+            const int r = c / CH, ch = c % CH;
+            const int key = key0 + r;
+            const bool ok = key < kv_len;
+            const size_t off = (size_t)(ok ? key : 0) * hidden + ch * 8;
+            cp_async16(Ks + (buf * ATT_KT + r) * LD + ch * 8, kbase + off, ok);
+            cp_async16(Vs + (buf * ATT_KT + r) * LD + ch * 8, vbase + off, ok);
+        }
+        cp_async_commit();
+    };
+
+    const bool active = warp * 16 < nq;
+    const int g = lane >> 2, tq = lane & 3;
+    const int qa = warp * 16 + g, qb = qa + 8;            // this thread's two query rows
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+    float o[D / 8][4];
+#pragma unroll
+    for (int j = 0; j < D / 8; j++) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+
+    if (t0 < t1) load_tile(t0, 0);
+    __syncthreads();                                       // Qs and pos_s visible
+    const int pa = pos_s[qa], pb = pos_s[qb];
+    uint32_t qf[D / 16][4];
+    if (active) {
+#pragma unroll
+        for (int kk = 0; kk < D / 16; kk++)
+            ldsm_x4(qf[kk], Qs + (warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + kk * 16 + (lane >> 4) * 8);
+    }
+    for (int t = t0; t < t1; t++) {
+        const int buf = (t - t0) & 1;
+        if (t + 1 < t1) { load_tile(t + 1, buf ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+        __syncthreads();
+        if (active) {
+            const __nv_bfloat16* Kt = Ks + buf * ATT_KT * LD;
+            const __nv_bfloat16* Vt = Vs + buf * ATT_KT * LD;
+            float s[ATT_KT / 8][4];
+#pragma unroll
+            for (int j = 0; j < ATT_KT / 8; j++) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+#pragma unroll
+            for (int kk = 0; kk < D / 16; kk++) {
+#pragma unroll
+                for (int jn = 0; jn < ATT_KT / 16; jn++) {
+                    uint32_t kb[4];
+                    ldsm_x4(kb, Kt + (jn * 16 + (lane & 7) + (lane >> 4) * 8) * LD + kk * 16 + ((lane >> 3) & 1) * 8);
+                    mma_bf16_16816(s[2 * jn], qf[kk], kb[0], kb[1]);
+                    mma_bf16_16816(s[2 * jn + 1], qf[kk], kb[2], kb[3]);
+                }
+            }
+            // scale, causal mask, running max
+            const int key0 = t * ATT_KT;
+            float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < ATT_KT / 8; j++) {
+                const int k0 = key0 + j * 8 + 2 * tq;
+                s[j][0] = (k0 <= pa) ? s[j][0] * scale_log2 : -INFINITY;
+                s[j][1] = (k0 + 1 <= pa) ? s[j][1] * scale_log2 : -INFINITY;
+                s[j][2] = (k0 <= pb) ? s[j][2] * scale_log2 : -INFINITY;
+                s[j][3] = (k0 + 1 <= pb) ? s[j][3] * scale_log2 : -INFINITY;
+                mx_a = fmaxf(mx_a, fmaxf(s[j][0], s[j][1]));
+                mx_b = fmaxf(mx_b, fmaxf(s[j][2], s[j][3]));
+            }
+            mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+            mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+            mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+            mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+            const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+            const float ua = mn_a == -INFINITY ? 0.f : mn_a, ub = mn_b == -INFINITY ? 0.f : mn_b;
+            const float ca = exp2f(m_a - ua), cb = exp2f(m_b - ub);
+            m_a = mn_a; m_b = mn_b;
+            float sa = 0.f, sb = 0.f;
+            uint32_t pf[ATT_KT / 16][4];
+#pragma unroll
+            for (int j = 0; j < ATT_KT / 8; j++) {
+                const float p0 = exp2f(s[j][0] - ua), p1 = exp2f(s[j][1] - ua);
+                const float p2 = exp2f(s[j][2] - ub), p3 = exp2f(s[j][3] - ub);
+                sa += p0 + p1;
+                sb += p2 + p3;
+                pf[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
+                pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+            }
+            l_a = l_a * ca + sa;
+            l_b = l_b * cb + sb;
+#pragma unroll
+            for (int j = 0; j < D / 8; j++) { o[j][0] *= ca; o[j][1] *= ca; o[j][2] *= cb; o[j][3] *= cb; }
+#pragma unroll
+            for (int kk = 0; kk < ATT_KT / 16; kk++) {
+#pragma unroll
+                for (int jn = 0; jn < D / 16; jn++) {
+                    uint32_t vb[4];
+                    ldsm_x4_t(vb, Vt + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + jn * 16 + (lane >> 4) * 8);
+                    mma_bf16_16816(o[2 * jn], pf[kk], vb[0], vb[1]);
+                    mma_bf16_16816(o[2 * jn + 1], pf[kk], vb[2], vb[3]);
+                }
+            }
+        }
+        __syncthreads();                                   // buffer may be refilled next round
+    }
+    if (active) {
+        // row sums live spread over the quad
+        l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+        l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+        l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+        l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+#pragma unroll
+        for (int half = 0; half < 2; half++) {
+            const int q = half ? qb : qa;
+            if (q < nq) {
+                const size_t base = ((size_t)(r0 + q) * H + hd) * n_splits + sp;
+                float* po = part_o + base * D;
+#pragma unroll
+                for (int j = 0; j < D / 8; j++)
+                    *reinterpret_cast<float2*>(po + j * 8 + 2 * tq) = make_float2(o[j][half * 2], o[j][half * 2 + 1]);
+                if (tq == 0) {
+                    part_ml[base * 2] = half ? m_b : m_a;
+                    part_ml[base * 2 + 1] = half ? l_b : l_a;
+                }
+            }
+        }
+    }
+}
+
+// out[row, head*D + e] = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), splits in ascending order.
+template <int D>
+__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_splits,
+                                    const int* __restrict__ row_pos, int hidden, __nv_bfloat16* __restrict__ out) {
+    const int r = blockIdx.x, hd = blockIdx.y, H = gridDim.y;
+    const int e = threadIdx.x;
+    if (e >= D) return;
+    __nv_bfloat16* dst = out + (size_t)r * hidden + hd * D + e;
+    if (row_pos[r] < 0) { *dst = __float2bfloat16_rn(0.f); return; }
+    const size_t base = ((size_t)r * H + hd) * n_splits;
+    float M = -INFINITY;
+    for (int s = 0; s < n_splits; s++) M = fmaxf(M, part_ml[(base + s) * 2]);
+    float num = 0.f, den = 0.f;
+    for (int s = 0; s < n_splits; s++) {
+        const float m = part_ml[(base + s) * 2];
+        if (m == -INFINITY) continue;
+        const float w = exp2f(m - M);
+        num += part_o[(base + s) * D + e] * w;
+        den += part_ml[(base + s) * 2 + 1] * w;
+    }
+    *dst = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+}
+
+}  // namespace rd

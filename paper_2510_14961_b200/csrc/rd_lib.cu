@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "../../include/rd.h"
+#include "rd_attn.cuh"
 #include "rd_gemm_tc.cuh"
 #include "rd_kernels.cuh"
 
@@ -231,6 +232,10 @@ struct rd_session {
     float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
     float* partial = nullptr;   // split-K partial sums of the tensor-core GEMM
     size_t partial_elems = 0;
+    float *att_o = nullptr, *att_ml = nullptr;   // split-KV partials of the windowed attention
+    int grp_rows = 0;           // rows per attention query group in the current pass
+    int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
+    int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128)
     void *act_h = nullptr, *act_2h = nullptr, *act_i = nullptr, *q_t = nullptr;
     void *Kc[3] = {nullptr, nullptr, nullptr}, *Vc[3] = {nullptr, nullptr, nullptr};
     TcAct t_act_h, t_act_2h, t_act_i;
@@ -348,6 +353,11 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         std::vector<int> ones(B, 1);
         if (e == cudaSuccess) e = cudaMemcpy(s->done, ones.data(), B * sizeof(int), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { rc = cuda_fail(e, "session init copies", __LINE__); break; }
+        if (c.dtype == RD_BF16 && (c.head_dim == 64 || c.head_dim == 96 || c.head_dim == 128)) {
+            if ((rc = s->mem.get(&s->att_o, R * c.n_heads * 8 * (size_t)c.head_dim * sizeof(float)))) break;
+            if ((rc = s->mem.get(&s->att_ml, R * c.n_heads * 8 * 2 * sizeof(float)))) break;
+            s->attn_path = 1;
+        }
         if (m->tc_ok) {
             s->partial_elems = tc_partial_elems(R, c);
             if ((rc = s->mem.get(&s->partial, s->partial_elems * sizeof(float)))) break;
@@ -407,6 +417,38 @@ template <typename T> struct Eng {
         return RD_OK;
     }
 
+    // Windowed flash-decode attention (bf16): groups of s->grp_rows rows share their sequence's KV.
+    template <int D>
+    static int attn_windowed_d(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
+        static bool attr_set = false;
+        if (!attr_set) {
+            CU(cudaFuncSetAttribute(attn_window_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<D>::SMEM));
+            attr_set = true;
+        }
+        const rd_config& c = s->m->cfg;
+        const int groups = (n_rows + s->grp_rows - 1) / s->grp_rows;
+        const int tiles = std::max(1, (s->ctx_max + ATT_KT - 1) / ATT_KT);
+        int ns = (2 * 148 + groups * c.n_heads - 1) / (groups * c.n_heads);
+        ns = std::max(1, std::min(std::min(ns, 8), tiles));
+        const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
+        attn_window_kernel<D><<<dim3(c.n_heads, groups, ns), 128, AttCfg<D>::SMEM, s->stream>>>(
+            (const bf16*)s->q_t, s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden,
+            scale_log2, ns, s->att_o, s->att_ml);
+        LAUNCHED(s);
+        attn_combine_kernel<D><<<dim3(n_rows, c.n_heads), D, 0, s->stream>>>(s->att_o, s->att_ml, ns, s->row_pos,
+                                                                              c.hidden, (bf16*)s->act_h);
+        LAUNCHED(s);
+        return RD_OK;
+    }
+    static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {
+        switch (s->m->cfg.head_dim) {
+            case 64: return attn_windowed_d<64>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            case 96: return attn_windowed_d<96>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            case 128: return attn_windowed_d<128>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            default: return RD_E_INVALID_ARG;
+        }
+    }
+
     // One transformer layer over the rows of the current row table, in place on x.
     static int layer(rd_session* s, int blk, int l, float* x, int n_rows) {
         const rd_config& c = s->m->cfg;
@@ -422,10 +464,19 @@ template <typename T> struct Eng {
                                                           c.head_dim, (T*)s->q_t, Kc, Vc, s->seq_stride);
         LAUNCHED(s);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
-        attn_row_kernel<T><<<dim3(n_rows, c.n_heads), 128, 0, s->stream>>>(
-            (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc, s->seq_stride, h, c.head_dim,
-            (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
-        LAUNCHED(s);
+        bool windowed = false;
+        if constexpr (sizeof(T) == 2) {
+            if (s->attn_path == 1 && s->grp_rows >= 1 && s->grp_rows <= ATT_QMAX) {
+                RD_TRY(attn_windowed(s, Kc, Vc, n_rows));
+                windowed = true;
+            }
+        }
+        if (!windowed) {
+            attn_row_kernel<T><<<dim3(n_rows, c.n_heads), 128, 0, s->stream>>>(
+                (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc, s->seq_stride, h, c.head_dim,
+                (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
+            LAUNCHED(s);
+        }
         bracket_close(s, br);
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, x, h, x, n_rows));
         rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g2, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
@@ -485,10 +536,14 @@ template <typename T> struct Eng {
         const int n = s->n_slots, h = c.hidden, B = s->sc.batch;
         // the leading edge of a wavefront advances by at most one position per step
         s->ctx_total = 0;
+        s->ctx_max = 1;
+        s->grp_rows = s->sc.max_window;
         for (int b = 0; b < B; b++)
             if (s->prefilled[b]) {
                 s->host_steps[b]++;
-                s->ctx_total += std::min(s->host_prompt_len[b] + s->host_steps[b], s->host_prompt_len[b] + s->sc.max_new_tokens);
+                const int ctx = std::min(s->host_prompt_len[b] + s->host_steps[b], s->host_prompt_len[b] + s->sc.max_new_tokens);
+                s->ctx_total += ctx;
+                s->ctx_max = std::max(s->ctx_max, ctx);
             }
         plan_rows_kernel<<<(n + 127) / 128, 128, 0, s->stream>>>(s->n_committed, s->win_len, s->done, B,
                                                                  s->sc.max_window, s->row_pos, s->row_seq,
@@ -528,6 +583,9 @@ template <typename T> struct Eng {
             // pass r+1: coda layers (fills the coda cache; no head).
             for (int c0 = 0; c0 < n && !rc; c0 += s->R) {
                 const int nr = std::min(s->R, n - c0);
+                s->grp_rows = ATT_QMAX;
+                s->ctx_max = c0 + nr;
+                s->ctx_total = c0 + nr;
                 fill_rows_kernel<<<(s->R + 127) / 128, 128, 0, s->stream>>>(seq, c0, nr, s->R, s->row_pos, s->row_seq);
                 s->stats.kernel_launches++;
                 float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
