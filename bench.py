@@ -41,6 +41,11 @@ WORKLOADS = {
                                   inner=1, eps=0.0, ar_r=32, prefill_r=32, temperature=0.0),
     "3p5b_b4_p8192_g1024_W32": dict(shape=rd_inputs.SHAPE_3P5B, bf16=True, batch=4, prompt=8192, gen=1024,
                                     window=32, inner=1, eps=0.0, ar_r=32, prefill_r=32, temperature=0.0),
+    # same GEMM and attention shapes as the 3.5B model with 1/1/1 layers and a small vocabulary:
+    # about 1.3 GB on the device, for ncu captures
+    "3p5b_layers111_v8192_p512_g64_W32": dict(shape=dict(rd_inputs.SHAPE_3P5B, n_prelude=1, n_core=1, n_coda=1, vocab=8192),
+                                              bf16=True, batch=1, prompt=512, gen=64, window=32, inner=1, eps=0.0,
+                                              ar_r=4, prefill_r=2, temperature=0.0),
 }
 DEFAULT_WORKLOAD = "3p5b_b1_p512_g256_W32"
 
