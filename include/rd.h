@@ -162,6 +162,30 @@ int rd_debug_force_tokens(rd_session* s, int32_t seq, int32_t first_pos, const i
 int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq,
                      int32_t pos0, int32_t n, float* dst);
 
+/* rd_debug_read_kv_noalloc -- rd_debug_read_kv for callers that must not allocate.  (The paper has
+ * no counterpart: this is a property of the library, not of the method.)
+ *
+ * Who needs it: a serving process that sized its KV caches to take all the device memory that was
+ * left, so a cudaMalloc of even a few megabytes fails; and a process that reads cache rows out while
+ * other sessions keep stepping on other streams, where cudaMalloc / cudaFree would stall the whole
+ * device for a moment.  rd_debug_read_kv takes a temporary float32 buffer from cudaMalloc on every
+ * call with a bf16 cache; this call stages through a fixed array that is part of the library image
+ * instead and calls no allocating routine.
+ *
+ * Arguments, layout of `dst` (host memory, float32 [n, hidden]) and results are those of
+ * rd_debug_read_kv: the values are bit-identical.  Differences:
+ *   - n * hidden may be at most 1,048,576 values (the staging array: 4 MiB, held by every device
+ *     that loads the library until the process exits).  More is refused with RD_E_CAPACITY and a
+ *     message in rd_last_cuda_error; nothing is read.
+ *   - The session's device must be the current device (RD_E_STATE otherwise).
+ *   - The first call on a device looks up the staging array's address on that device
+ *     (cudaGetSymbolAddress) and remembers it; make that first call before any stream capture.
+ *   - All calls on one device share the one staging array.  A call overwrites every value it later
+ *     copies out, so the previous call's contents never show; but two calls that overlap in time on
+ *     the same device (two host threads, two sessions) race on it: serialise them. */
+int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq,
+                             int32_t pos0, int32_t n, float* dst);
+
 /* rd_stats -- counters since session creation (host pointer out). */
 int rd_stats(rd_session* s, rd_stats_t* out);
 

@@ -17,7 +17,7 @@ RD_DBG_LATENTS, RD_DBG_DELTA, RD_DBG_DRAFTS, RD_DBG_LOGITS, RD_DBG_EMBED = 0, 1,
 EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_prefill", "rd_ar_step",
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
-           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read"]
+           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc"]
 
 
 class RdConfig(C.Structure):
@@ -75,6 +75,7 @@ def lib():
         L.rd_debug_read.argtypes = [vp, i32, i32, vp, C.c_size_t]
         L.rd_debug_force_tokens.argtypes = [vp, i32, i32, vp, i32]
         L.rd_debug_read_kv.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
+        L.rd_debug_read_kv_noalloc.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
         L.rd_stats.argtypes = [vp, C.POINTER(RdStats)]
         L.rd_set_gemm_path.argtypes = [vp, i32]
         L.rd_profile_enable.argtypes = [vp, i32]
@@ -204,6 +205,15 @@ class Session:
         out = np.empty((n, self.model.cfg.hidden), dtype=np.float32)
         _check(lib().rd_debug_read_kv(self.handle, block, layer, which, seq, pos0, n, out.ctypes.data),
                "rd_debug_read_kv")
+        return out
+
+    def read_kv_noalloc(self, block, layer, which, seq, pos0, n):
+        """read_kv through the library's fixed staging array: no device allocation is made.  For
+        callers that cannot allocate (device memory fully committed, or other streams must not be
+        stalled); at most 1,048,576 values per call, calls on one device must not overlap."""
+        out = np.empty((n, self.model.cfg.hidden), dtype=np.float32)
+        _check(lib().rd_debug_read_kv_noalloc(self.handle, block, layer, which, seq, pos0, n, out.ctypes.data),
+               "rd_debug_read_kv_noalloc")
         return out
 
     def stats(self):

@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -770,6 +771,69 @@ extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int
     if (e == cudaSuccess) e = cudaMemcpy(dst, tmp, cnt * 4, cudaMemcpyDeviceToHost);
     cudaFree(tmp);
     if (e != cudaSuccess) return cuda_fail(e, "read_kv", __LINE__);
+    return RD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// rd_debug_read_kv_noalloc: the K/V read-out without any allocation.
+//
+// rd_debug_read_kv widens bf16 cache rows to float32 in a temporary device buffer that it obtains
+// from cudaMalloc and returns with cudaFree.  Here the temporary is a fixed array that is part of
+// the library image: every device that loads the library holds RD_KV_STAGE_ELEMS floats (4 MiB)
+// until the process exits.  In host code `g_kv_stage` is only a handle for the runtime, not an
+// address a kernel can use; the address on a given device comes from cudaGetSymbolAddress, asked
+// once per device with that device current and remembered in g_kv_stage_dev.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t RD_KV_STAGE_ELEMS = (size_t)1 << 20;
+static __device__ __align__(256) float g_kv_stage[RD_KV_STAGE_ELEMS];
+constexpr int RD_MAX_DEVICES = 64;
+static float* g_kv_stage_dev[RD_MAX_DEVICES];
+static std::mutex g_kv_stage_mutex;
+
+// Device address of g_kv_stage on the current device (which must be `device`).
+static int kv_stage_address(int device, float** out) {
+    if (device < 0 || device >= RD_MAX_DEVICES) return RD_E_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_kv_stage_mutex);
+    if (!g_kv_stage_dev[device]) {
+        float* p = nullptr;
+        CU(cudaGetSymbolAddress((void**)&p, g_kv_stage));
+        if (!p) return RD_E_CUDA;
+        g_kv_stage_dev[device] = p;
+    }
+    *out = g_kv_stage_dev[device];
+    return RD_OK;
+}
+
+extern "C" int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq,
+                                        int32_t pos0, int32_t n, float* dst) {
+    if (!s || !dst || block < 0 || block > 2 || (which != 0 && which != 1) || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    const rd_config& c = s->m->cfg;
+    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 + n > s->sc.max_context) return RD_E_INVALID_ARG;
+    const size_t cnt = (size_t)n * c.hidden;
+    if (cnt > RD_KV_STAGE_ELEMS) {
+        snprintf(g_cuda_err, sizeof g_cuda_err,
+                 "rd_debug_read_kv_noalloc: %zu values asked for, the fixed staging array holds %zu (n * hidden too large)",
+                 cnt, RD_KV_STAGE_ELEMS);
+        return RD_E_CAPACITY;
+    }
+    int dev = -1;
+    CU(cudaGetDevice(&dev));
+    if (dev != s->m->device) return RD_E_STATE;   // the session's device must be current
+    RD_TRY(rd_sync(s));
+    if (n == 0) return RD_OK;
+    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride + (size_t)pos0 * c.hidden;
+    const char* src = (const char*)(which ? s->Vc[block] : s->Kc[block]) + off * s->m->esz;
+    if (c.dtype == RD_F32) {                      // float32 cache: no staging needed at all
+        CU(cudaMemcpy(dst, src, cnt * 4, cudaMemcpyDeviceToHost));
+        return RD_OK;
+    }
+    float* stage = nullptr;
+    RD_TRY(kv_stage_address(dev, &stage));
+    // every element of stage[0..cnt) is overwritten: nothing of an earlier call can show through
+    widen_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, stage, cnt);
+    CU(cudaGetLastError());
+    CU(cudaStreamSynchronize(s->stream));
+    CU(cudaMemcpy(dst, stage, cnt * 4, cudaMemcpyDeviceToHost));
     return RD_OK;
 }
 
