@@ -206,6 +206,11 @@ int rd_profile_read(rd_session* s, rd_profile_t* out);
  * GEMMs where the shape allows.  For measurement and parity tests. */
 int rd_set_gemm_path(rd_session* s, int32_t path);
 
+/* rd_set_launch_chaining -- 1 (default): the kernels of a step are launched as a programmatic-
+ * dependent-launch chain (each may start, and prefetch weights, while its predecessor finishes);
+ * 0: ordinary stream-ordered launches.  Results are identical; for measurement and tests. */
+int rd_set_launch_chaining(rd_session* s, int32_t on);
+
 const char* rd_strerror(int code);
 /* Text of the last CUDA error this library saw on the calling thread's most recent failing call
  * (static storage, never NULL). */

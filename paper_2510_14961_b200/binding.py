@@ -17,7 +17,7 @@ RD_DBG_LATENTS, RD_DBG_DELTA, RD_DBG_DRAFTS, RD_DBG_LOGITS, RD_DBG_EMBED = 0, 1,
 EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_prefill", "rd_ar_step",
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
-           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc"]
+           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining"]
 
 
 class RdConfig(C.Structure):
@@ -78,6 +78,7 @@ def lib():
         L.rd_debug_read_kv_noalloc.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp]
         L.rd_stats.argtypes = [vp, C.POINTER(RdStats)]
         L.rd_set_gemm_path.argtypes = [vp, i32]
+        L.rd_set_launch_chaining.argtypes = [vp, i32]
         L.rd_profile_enable.argtypes = [vp, i32]
         L.rd_profile_read.argtypes = [vp, C.POINTER(RdProfile)]
         L.rd_strerror.argtypes = [C.c_int]
@@ -223,6 +224,9 @@ class Session:
 
     def set_gemm_path(self, path):
         _check(lib().rd_set_gemm_path(self.handle, path), "rd_set_gemm_path")
+
+    def set_launch_chaining(self, on):
+        _check(lib().rd_set_launch_chaining(self.handle, 1 if on else 0), "rd_set_launch_chaining")
 
     def profile_enable(self, on=True):
         _check(lib().rd_profile_enable(self.handle, 1 if on else 0), "rd_profile_enable")

@@ -15,6 +15,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "rd_common.cuh"
+
 namespace rd {
 
 constexpr int ATT_KT = 64;          // keys per tile
@@ -71,6 +73,7 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     __nv_bfloat16* Vs = Ks + 2 * ATT_KT * LD;             // [2][KT][LD]
     int* pos_s = (int*)(Vs + 2 * ATT_KT * LD);
 
+    pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int hd = blockIdx.x, H = gridDim.x, sp = blockIdx.z;
     const int r0 = blockIdx.y * rows_per_group;
@@ -218,6 +221,7 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
 template <int D>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_splits,
                                     const int* __restrict__ row_pos, int hidden, __nv_bfloat16* __restrict__ out) {
+    pdl_enter();
     const int r = blockIdx.x, hd = blockIdx.y, H = gridDim.y;
     const int e = threadIdx.x;
     if (e >= D) return;

@@ -1,0 +1,36 @@
+// Pieces every kernel file of the library uses: programmatic dependent launch.
+//
+// The kernels of one step form a chain on one stream.  Each is launched with the programmatic
+// stream-serialization attribute: it may start while its predecessor still runs, must call
+// pdl_wait() before it reads anything an earlier kernel wrote or writes anything an earlier kernel
+// may still read, and calls pdl_trigger() at its start so that its own successor can be scheduled
+// early.  pdl_wait() returns once the predecessor has completed and its writes are visible; as
+// every kernel of the chain waits before it finishes, completion is transitive along the chain.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace rd {
+
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Start of a kernel that has nothing useful to do before its inputs are ready.
+__device__ __forceinline__ void pdl_enter() { pdl_trigger(); pdl_wait(); }
+
+// Launch `kern` on `st` as a link of the chain (`chained` false: an ordinary launch).
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                         bool chained, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+}  // namespace rd

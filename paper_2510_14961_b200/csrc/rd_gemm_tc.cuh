@@ -1,17 +1,36 @@
 // Weight-streaming GEMM on the 5th-generation tensor cores (tcgen05 + TMEM, operands by TMA).
 //
-//   Y[r, o] = sum_k X[r, k] * W[o, k]  (+ resid[r, o]),   X: [rows, K] bf16,  W: [n_out, K] bf16
+//   acc[r, o] = sum_k X[r, k] * W[o, k],   X: [rows, K] bf16,  W: [n_out, K] bf16
 //
-// The W positions in flight share the weights, so one step is a dense contraction; at W <= 256 rows
+// The W positions in flight share the weights, so one step is a dense contraction; below ~250 rows
 // it is bound by streaming W from HBM once.  Mapping: the WEIGHT tile is the UMMA M operand
 // (128 output features x 64 k), the activation rows are the N operand (16..256 rows x 64 k), both
 // K-major with the 128-byte swizzle TMA writes; the accumulator D[feature, row] lives in TMEM
-// (128 lanes x BN columns, fp32).  One CTA computes one (feature tile, row tile, K range) unit:
+// (128 lanes x BN columns, fp32, two buffers).
+//
+// Persistent stream-K schedule: the (feature tile, row tile, k-block) units are numbered tile by
+// tile and cut into one contiguous share per CTA (one CTA per SM), so every SM streams the same
+// number of weight bytes through one long-lived ring whatever n_out is.  A share is a list of
+// segments (tile, k-block range):
 //   warp 0 / lane 0   TMA producer: fills a ring of STAGES {A,B} stages, mbarrier complete_tx
 //   warp 1 / lane 0   issues tcgen05.mma (4 per stage, K = 16 each); tcgen05.commit frees the stage
-//   warps 0-3         epilogue: tcgen05.ld of their 32 TMEM lanes, coalesced stores along features
-// Split-K units write fp32 partials [split][row][feature]; a second kernel adds them in split order
-// (no float atomics: results are bit-reproducible).
+//                     and, at the end of a segment, publishes the accumulator buffer
+//   warps 2-5         epilogue: tcgen05.ld of their 32 TMEM lanes; the next segment's MMAs run
+//                     meanwhile in the other accumulator buffer
+// A segment that covers the whole K range is finished from TMEM.  Otherwise its fp32 partial goes
+// to a scratch slot and a per-tile counter is bumped; the CTA that brings the counter to the
+// number of segments of the tile adds all partials IN K ORDER and finishes the tile.  No float
+// atomics and no order that depends on timing: results are bit-reproducible.  Nobody waits for
+// another CTA.
+//
+// Finishing a tile applies the fused epilogue: store (+ residual); SwiGLU on interleaved gate/up
+// features -> bf16; rotary embedding on q,k -> q buffer and the K/V cache entries of the rows.
+//
+// Programmatic dependent launch: the kernel lets its successor start at once, and itself starts
+// while its predecessor still runs: it sets up, prefetches the first weight stages (weights do not
+// depend on earlier kernels), and only then waits for the predecessor before touching activations
+// or outputs.
+//
 // Every wait on an mbarrier is bounded; on time-out the kernel raises a status word, drains the
 // copies it issued, frees its TMEM and returns.
 #pragma once
@@ -23,13 +42,16 @@
 #include <algorithm>
 
 #include "../../include/rd.h"
+#include "rd_common.cuh"
 
 namespace rd {
 
 constexpr int TC_BM = 128;       // output features per tile (UMMA M)
 constexpr int TC_BK = 64;        // k per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int TC_MAX_SPLITS = 8;
+constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
+
+enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_QKV = 2 };
 
 struct TcWeight {
     CUtensorMap map;
@@ -101,6 +123,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -151,6 +176,10 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16), stored as
 // TMA's 128-byte swizzle writes them: 8-row groups 1024 bytes apart (stride offset), descriptor
 // version 1, layout type SWIZZLE_128B.  Successive K = 16 slices start 32 bytes further on.
@@ -166,219 +195,354 @@ template <int BN> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;                 // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = BN <= 16 ? 6 : BN <= 32 ? 5 : BN <= 64 ? 4 : BN <= 128 ? 3 : 4;
+    // about 200 KB of ring per CTA (one CTA per SM): enough bytes in flight to cover HBM latency at
+    // full bandwidth, and a CTA that starts early under programmatic dependent launch prefetches
+    // that much of its weights while the kernels before it finish
+    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 12 ? 12 : (200 * 1024) / STAGE_BYTES;
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
-    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    static constexpr int ACC_COLS = BN < 32 ? 32 : BN;                // columns of one accumulator buffer
+    static constexpr int TMEM_COLS = 2 * ACC_COLS;                    // power of two, 64..512
+};
+
+// What finishing a tile does with acc[r, o].
+struct TcEpilogue {
+    int mode;
+    // TC_EPI_STORE: Y[r, o] = acc (+ resid[r, o])
+    float* Y; size_t ldy; const float* resid; size_t ldr;
+    // TC_EPI_SWIGLU: features come in groups of 32 = 16 gate, then the 16 matching up features;
+    // act[r, j] = silu(gate_j) * up_j, j < inner
+    __nv_bfloat16* act; size_t lda; int inner;
+    // TC_EPI_QKV: o in [0, 3 hidden) = q | k | v.  Rotary embedding on adjacent pairs of q and k with
+    // the row's position; q -> q_t[r], k and v -> the row's own cache entry.
+    __nv_bfloat16 *q_t, *Kc, *Vc; size_t seq_stride; int hidden, head_dim;
+    const int *row_pos, *row_seq; const float *cos_t, *sin_t;
 };
 
 struct TcParams {
     int K, n_out, n_rows;
-    int kb_total, kb_per_split, n_splits;
-    float* Y; size_t ldy;             // used when n_splits == 1
-    const float* resid;
-    float* partial;                   // [split][rows_pad][n_out] when n_splits > 1
-    int rows_pad;
+    int kb;                    // k-blocks per tile
+    int n_tiles_m, n_tiles_n;
+    long long units;           // n_tiles_m * n_tiles_n * kb
+    int per;                   // units per CTA
+    float* scratch;            // [2 * gridDim.x][BN][128] partial sums
+    int* counters;             // [tiles] arrivals of partial segments; zero between launches
     int* status;
+    TcEpilogue e;
 };
 
+// Finish 16 rows (columns c0..c0+15 of the accumulator) of this thread's output feature.
 template <int BN>
-__global__ void __launch_bounds__(128)
+__device__ __forceinline__ void tc_finish_chunk(const TcParams& p, int m0, int n0, int c0, int quad, int lane, const float* v) {
+    const TcEpilogue& e = p.e;
+    const int f = quad * 32 + lane;
+    const int m = m0 + f;
+    if (e.mode == TC_EPI_STORE) {
+        if (m < p.n_out) {
+#pragma unroll
+            for (int j = 0; j < 16; j++) {
+                const int r = n0 + c0 + j;
+                if (r < p.n_rows) e.Y[(size_t)r * e.ldy + m] = e.resid ? e.resid[(size_t)r * e.ldr + m] + v[j] : v[j];
+            }
+        }
+    } else if (e.mode == TC_EPI_SWIGLU) {
+        const int jf = (m0 >> 1) + quad * 16 + (lane & 15);
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const float up = __shfl_xor_sync(0xffffffffu, v[j], 16);
+            const int r = n0 + c0 + j;
+            if (lane < 16 && jf < e.inner && r < p.n_rows) {
+                const float g = v[j];
+                e.act[(size_t)r * e.lda + jf] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * up);
+            }
+        }
+    } else {
+        const int sec = m / e.hidden, mm = m - sec * e.hidden;
+        const int half = e.head_dim >> 1;
+        const int i = (mm % e.head_dim) >> 1;
+        const bool odd = (m & 1) != 0;
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
+            const int r = n0 + c0 + j;
+            if (m >= p.n_out || r >= p.n_rows) continue;
+            const int pos = e.row_pos[r];
+            if (pos < 0) continue;
+            float out = v[j];
+            if (sec < 2) {
+                const float c = e.cos_t[(size_t)pos * half + i], s = e.sin_t[(size_t)pos * half + i];
+                out = odd ? other * s + v[j] * c : v[j] * c - other * s;
+            }
+            const __nv_bfloat16 o16 = __float2bfloat16_rn(out);
+            if (sec == 0) {
+                e.q_t[(size_t)r * e.hidden + mm] = o16;
+            } else {
+                __nv_bfloat16* dst = (sec == 1 ? e.Kc : e.Vc) + (size_t)e.row_seq[r] * e.seq_stride + (size_t)pos * e.hidden;
+                dst[mm] = o16;
+            }
+        }
+    }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const TcParams p) {
     using C = TcCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* full = (uint64_t*)(smem + C::STAGES * C::STAGE_BYTES);
     uint64_t* empty = full + C::STAGES;
-    uint64_t* accum = empty + C::STAGES;
-    uint32_t* tmem_slot = (uint32_t*)(accum + 1);
+    uint64_t* acc_full = empty + C::STAGES;     // [2]
+    uint64_t* acc_empty = acc_full + 2;         // [2]
+    uint64_t* epi_bar = acc_empty + 2;          // the 128 epilogue threads meet here (bounded waits)
+    uint32_t* tmem_slot = (uint32_t*)(epi_bar + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile uint32_t* last_flag = tmem_slot + 2;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * TC_BM;
-    const int split = blockIdx.y;
-    const int n0 = blockIdx.z * BN;
-    const int kb0 = split * p.kb_per_split;
-    const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-    const int nkb = kb1 - kb0;
+    const long long u0 = (long long)blockIdx.x * p.per;
+    const long long u1 = min(p.units, u0 + p.per);
+    pdl_trigger();
+    if (u0 >= u1) { pdl_wait(); return; }       // no share for this CTA (uniform for the whole CTA)
+    const int n_units = (int)(u1 - u0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        mbar_init(accum, 1);
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        mbar_init(epi_bar, 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
 
-    if (threadIdx.x == 0) {
-        // ---- TMA producer ----
-        int issued = 0;
-        for (int i = 0; i < nkb; i++) {
-            const int s = i % C::STAGES;
-            if (i >= C::STAGES && !mbar_wait(&empty[s], ((i / C::STAGES) - 1) & 1)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
-            mbar_expect_tx(&full[s], C::STAGE_BYTES);
-            uint8_t* a = smem + s * C::STAGE_BYTES;
-            tma_load_2d(a, &tmap_w, (kb0 + i) * TC_BK, m0, &full[s]);
-            tma_load_2d(a + C::A_BYTES, &tmap_x, (kb0 + i) * TC_BK, n0, &full[s]);
-            issued = i + 1;
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            // Weights do not depend on the previous kernel: the first ring of A tiles is requested
+            // before the dependency wait, the matching B tiles after it.
+            const int pre = min(n_units, C::STAGES);
+            for (int i = 0; i < pre; i++) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                mbar_expect_tx(&full[i], C::STAGE_BYTES);
+                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM, &full[i]);
+            }
+            pdl_wait();
+            for (int i = 0; i < pre; i++) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[i]);
+            }
+            int issued = pre;
+            for (int i = pre; i < n_units; i++) {
+                const int s = i % C::STAGES;
+                if (*abort_flag || !mbar_wait(&empty[s], ((i / C::STAGES) - 1) & 1)) { *abort_flag = 1; break; }
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                mbar_expect_tx(&full[s], C::STAGE_BYTES);
+                uint8_t* a = smem + s * C::STAGE_BYTES;
+                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM, &full[s]);
+                tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[s]);
+                issued = i + 1;
+            }
+            if (*abort_flag) {
+                // drain: every stage this thread armed must land before the CTA's memory is released
+                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1);
+            }
+        } else {
+            pdl_wait();
         }
-        if (*abort_flag) {
-            // drain: every stage this thread armed must land before the CTA's memory is released
-            for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1);
-        }
-    } else if (threadIdx.x == 32) {
-        // ---- MMA issuer ----
-        constexpr uint32_t idesc = umma_idesc(BN);
-        bool ok = true;
-        for (int i = 0; i < nkb && ok; i++) {
-            const int s = i % C::STAGES;
-            if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1)) { *abort_flag = 1; ok = false; break; }
-            tc_fence_after();
-            const uint32_t a = smem_u32(smem + s * C::STAGE_BYTES);
-            const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
+    } else {
+        if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+        tc_fence_before();
+        named_bar_sync(1, TC_THREADS - 32);
+        tc_fence_after();
+        const uint32_t tmem_base = *tmem_slot;
+        pdl_wait();
+        if (warp == 1) {
+            if (lane == 0) {
+                // ---- MMA issuer ----
+                constexpr uint32_t idesc = umma_idesc(BN);
+                int i = 0, seg = 0;
+                bool ok = true;
+                while (i < n_units && ok) {
+                    const long long u = u0 + i;
+                    const int ka = (int)(u % p.kb);
+                    const int len = min(p.kb - ka, n_units - i);
+                    const int buf = seg & 1;
+                    if (seg >= 2 && !mbar_wait(&acc_empty[buf], ((seg >> 1) - 1) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d = tmem_base + (uint32_t)(buf * C::ACC_COLS);
+                    for (int j = 0; j < len; j++, i++) {
+                        const int s = i % C::STAGES;
+                        if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a = smem_u32(smem + s * C::STAGE_BYTES);
+                        const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
 #pragma unroll
-            for (int k = 0; k < TC_BK / 16; k++)
-                umma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (i | k) ? 1u : 0u);
-            umma_commit(&empty[s]);          // stage reusable once these MMAs have read it
-        }
-        umma_commit(accum);                  // accumulator complete (arrives even after an abort)
-    }
-    // ---- epilogue: all four warps ----
-    __syncwarp();
-    const bool done = mbar_wait(accum, 0);
-    tc_fence_after();
-    if (!done) *abort_flag = 1;
-    __syncthreads();
-    if (*abort_flag) {
-        if (threadIdx.x == 0) atomicExch(p.status, 1);
-    } else if (nkb > 0) {
-        const int m = m0 + warp * 32 + lane;              // TMEM lane = output feature
+                        for (int k = 0; k < TC_BK / 16; k++)
+                            umma_bf16(d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (j | k) ? 1u : 0u);
+                        umma_commit(&empty[s]);          // stage reusable once these MMAs have read it
+                    }
+                    if (!ok) break;
+                    umma_commit(&acc_full[buf]);         // this segment's sums are complete
+                    seg++;
+                }
+                if (!ok) *abort_flag = 1;
+            }
+        } else {
+            // ---- epilogue warps 2..5: TMEM lane quadrant = warp % 4 ----
+            const int quad = warp & 3;
+            const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+            int i = 0, seg = 0;
+            uint32_t epi_phase = 0;
+            bool ok = true;
+            // all 128 epilogue threads arrive, then wait for the phase: false if someone never came
+            auto epi_sync = [&]() -> bool {
+                mbar_arrive(epi_bar);
+                const bool done = mbar_wait(epi_bar, epi_phase & 1);
+                epi_phase++;
+                return done;
+            };
+            while (i < n_units && ok) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), ka = (int)(u % p.kb);
+                const int len = min(p.kb - ka, n_units - i);
+                const int buf = seg & 1;
+                const int m0 = (tile % p.n_tiles_m) * TC_BM, n0 = (tile / p.n_tiles_m) * BN;
+                const bool whole = (ka == 0 && len == p.kb);
+                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg >> 1) & 1)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_COLS);
+                // first segment of the share -> slot 2g, a later partial one (the last) -> 2g + 1
+                float* slot = p.scratch + ((size_t)blockIdx.x * 2 + (i == 0 ? 0 : 1)) * (size_t)(BN * TC_BM);
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-            uint32_t v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, v);
-            if (m < p.n_out) {
+                for (int c = 0; c < BN; c += 16) {
+                    uint32_t raw[16];
+                    tmem_ld16(t + (uint32_t)c, raw);
+                    float v[16];
 #pragma unroll
-                for (int j = 0; j < 16; j++) {
-                    const int r = n0 + c + j;
-                    if (r < p.n_rows) {
-                        const float acc = __uint_as_float(v[j]);
-                        if (p.n_splits == 1) {
-                            const size_t o = (size_t)r * p.ldy + m;
-                            p.Y[o] = p.resid ? p.resid[o] + acc : acc;
-                        } else {
-                            p.partial[((size_t)split * p.rows_pad + r) * p.n_out + m] = acc;
-                        }
+                    for (int j = 0; j < 16; j++) v[j] = __uint_as_float(raw[j]);
+                    if (whole) {
+                        tc_finish_chunk<BN>(p, m0, n0, c, quad, lane, v);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; j++) slot[(size_t)(c + j) * TC_BM + quad * 32 + lane] = v[j];
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);     // accumulator buffer may be overwritten
+                if (!whole) {
+                    // publish the partial; the CTA that completes the tile's count finishes it
+                    const long long t_lo = (long long)tile * p.kb;
+                    const int g_lo = (int)(t_lo / p.per), g_hi = (int)((t_lo + p.kb - 1) / p.per);
+                    __threadfence();
+                    if (!epi_sync()) { ok = false; break; }
+                    if (et == 0) {
+                        const int old = atomicAdd(&p.counters[tile], 1);
+                        const bool last = old == g_hi - g_lo;
+                        if (last) p.counters[tile] = 0;          // ready for the next launch
+                        *last_flag = last ? 1u : 0u;
+                    }
+                    if (!epi_sync()) { ok = false; break; }
+                    if (*last_flag) {
+                        __threadfence();
+#pragma unroll 1
+                        for (int c = 0; c < BN; c += 16) {
+                            float v[16];
+#pragma unroll
+                            for (int j = 0; j < 16; j++) v[j] = 0.f;
+                            for (int g = g_lo; g <= g_hi; g++) {          // ascending k
+                                const int first_tile = (int)(((long long)g * p.per) / p.kb);
+                                const float* sl = p.scratch + ((size_t)g * 2 + (first_tile == tile ? 0 : 1)) * (size_t)(BN * TC_BM);
+#pragma unroll
+                                for (int j = 0; j < 16; j++) v[j] += __ldcg(sl + (size_t)(c + j) * TC_BM + quad * 32 + lane);
+                            }
+                            tc_finish_chunk<BN>(p, m0, n0, c, quad, lane, v);
+                        }
+                    }
+                    // (last_flag is next written after the next segment's first meeting, which every
+                    // thread reaches only after it has read the flag here)
+                }
+                i += len;
+                seg++;
             }
+            if (!ok) *abort_flag = 1;
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, C::TMEM_COLS);
-}
-
-// Y[r, o] = resid[r, o] + sum_s partial[s][r][o], s ascending.
-__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int n_splits, int rows_pad, int n_rows,
-                                     int n_out, float* __restrict__ Y, size_t ldy, const float* __restrict__ resid) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= (size_t)n_rows * n_out) return;
-    const size_t r = i / n_out, o = i % n_out;
-    float acc = 0.f;
-    for (int s = 0; s < n_splits; s++) acc += partial[((size_t)s * rows_pad + r) * n_out + o];
-    const size_t y = r * ldy + o;
-    Y[y] = resid ? resid[y] + acc : acc;
+    if (*abort_flag && threadIdx.x == 0) atomicExch(p.status, 1);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(*tmem_slot, C::TMEM_COLS);
+    }
 }
 
 static inline int tc_pick_bn(int n_rows) { return n_rows <= 16 ? 0 : n_rows <= 32 ? 1 : n_rows <= 64 ? 2 : n_rows <= 128 ? 3 : 4; }
 
-// Number of K splits for a GEMM: enough (feature tile x row tile x split) units to fill the 148
-// SMs twice over, never fewer than 8 k-blocks per unit.
-static inline void tc_plan(int K, int n_out, int n_rows, int* bn_idx, int* n_splits, int* kb_per_split, int* kb_total) {
-    *bn_idx = tc_pick_bn(n_rows);
-    const int bn = 16 << *bn_idx;
-    const int tiles = ((n_out + TC_BM - 1) / TC_BM) * ((n_rows + bn - 1) / bn);
-    const int kb = (K + TC_BK - 1) / TC_BK;
-    int s = (2 * 148 + tiles - 1) / tiles;
-    s = s > TC_MAX_SPLITS ? TC_MAX_SPLITS : s;
-    const int max_by_k = kb / 8 > 1 ? kb / 8 : 1;
-    s = s > max_by_k ? max_by_k : s;
-    const int per = (kb + s - 1) / s;
-    *kb_per_split = per;
-    *n_splits = (kb + per - 1) / per;
-    *kb_total = kb;
+struct TcPlan {
+    int bn_idx, bn, kb, n_tiles_m, n_tiles_n, per, grid;
+    long long units;
+};
+// One CTA per SM; every CTA gets `per` consecutive units (the last ones possibly fewer).
+static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms) {
+    TcPlan pl;
+    pl.bn_idx = tc_pick_bn(n_rows);
+    pl.bn = 16 << pl.bn_idx;
+    pl.kb = (K + TC_BK - 1) / TC_BK;
+    pl.n_tiles_m = (n_out + TC_BM - 1) / TC_BM;
+    pl.n_tiles_n = (n_rows + pl.bn - 1) / pl.bn;
+    pl.units = (long long)pl.n_tiles_m * pl.n_tiles_n * pl.kb;
+    const long long g = std::min<long long>(n_sms, pl.units);
+    pl.per = (int)((pl.units + g - 1) / g);
+    pl.grid = (int)((pl.units + pl.per - 1) / pl.per);
+    return pl;
 }
 
-// Scratch the split-K partials of this model need at `rows` rows.
-static inline size_t tc_partial_elems(size_t rows, const rd_config& c) {
-    const int shapes[6][2] = {{c.hidden, 3 * c.hidden}, {c.hidden, c.hidden}, {c.hidden, 2 * c.mlp_inner},
-                              {c.mlp_inner, c.hidden}, {2 * c.hidden, c.hidden}, {c.hidden, c.vocab}};
-    size_t need = 16;
-    for (int n = 1; n <= (int)rows; n = n < 16 ? 16 : n * 2) {
-        const int nr = n > (int)rows ? (int)rows : n;
-        for (auto& sh : shapes) {
-            int bi, ns, per, kb;
-            tc_plan(sh[0], sh[1], nr, &bi, &ns, &per, &kb);
-            const int bn = 16 << bi;
-            const size_t rows_pad = (size_t)((nr + bn - 1) / bn) * bn;
-            if (ns > 1) need = std::max(need, (size_t)ns * rows_pad * sh[1]);
-        }
-        if (n >= (int)rows) break;
-    }
-    return need;
+// Scratch (floats) for the partial sums and counters (ints) a session with `rows` rows needs.
+static inline size_t tc_scratch_elems(size_t rows, int n_sms) {
+    const int bn = 16 << tc_pick_bn((int)std::min<size_t>(rows, 256));
+    return (size_t)2 * n_sms * bn * TC_BM;
+}
+static inline size_t tc_counter_elems(size_t rows, int max_n_out) {
+    return ((size_t)max_n_out / TC_BM + 1) * (rows / 16 + 1);
 }
 
 template <int BN>
-static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, dim3 grid) {
+static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, int grid, bool chained) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM) != cudaSuccess)
             return RD_E_CUDA;
         attr_set = true;
     }
-    gemm_tc_kernel<BN><<<grid, 128, TcCfg<BN>::SMEM, st>>>(mw, mx, p);
-    return cudaGetLastError() == cudaSuccess ? RD_OK : RD_E_CUDA;
+    return launch_chained(gemm_tc_kernel<BN>, dim3(grid), dim3(TC_THREADS), TcCfg<BN>::SMEM, st, chained, mw, mx, p) == cudaSuccess
+               ? RD_OK : RD_E_CUDA;
 }
 
-// Returns RD_E_INVALID_ARG when the shape is not taken (caller falls back to the SIMT kernel).
-static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, float* Y, size_t ldy,
-                          const float* resid, int n_rows, float* partial, size_t partial_elems, int* status,
-                          uint64_t* launches) {
+// Returns RD_E_INVALID_ARG when the shape is not taken (caller falls back to the SIMT kernels).
+static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
+                          const TcEpilogue& epi, float* scratch, size_t scratch_elems, int* counters,
+                          size_t counter_elems, int n_sms, int* status, bool chained) {
     if (ta.K != K || tw.K != K || tw.n_out != n_out || n_rows < 1 || n_rows > ta.rows) return RD_E_INVALID_ARG;
+    const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms);
+    if ((size_t)2 * pl.grid * pl.bn * TC_BM > scratch_elems) return RD_E_INVALID_ARG;
+    if ((size_t)pl.n_tiles_m * pl.n_tiles_n > counter_elems) return RD_E_INVALID_ARG;
     TcParams p;
-    int bi;
-    tc_plan(K, n_out, n_rows, &bi, &p.n_splits, &p.kb_per_split, &p.kb_total);
-    const int bn = 16 << bi;
-    const int n_tiles = (n_rows + bn - 1) / bn;
     p.K = K; p.n_out = n_out; p.n_rows = n_rows;
-    p.Y = Y; p.ldy = ldy; p.resid = resid; p.partial = partial; p.status = status;
-    p.rows_pad = n_tiles * bn;
-    if (p.n_splits > 1 && (size_t)p.n_splits * p.rows_pad * n_out > partial_elems) return RD_E_INVALID_ARG;
-    const dim3 grid((n_out + TC_BM - 1) / TC_BM, p.n_splits, n_tiles);
-    int rc;
-    switch (bi) {
-        case 0: rc = tc_launch<16>(st, tw.map, ta.map[0], p, grid); break;
-        case 1: rc = tc_launch<32>(st, tw.map, ta.map[1], p, grid); break;
-        case 2: rc = tc_launch<64>(st, tw.map, ta.map[2], p, grid); break;
-        case 3: rc = tc_launch<128>(st, tw.map, ta.map[3], p, grid); break;
-        default: rc = tc_launch<256>(st, tw.map, ta.map[4], p, grid); break;
+    p.kb = pl.kb; p.n_tiles_m = pl.n_tiles_m; p.n_tiles_n = pl.n_tiles_n;
+    p.units = pl.units; p.per = pl.per;
+    p.scratch = scratch; p.counters = counters; p.status = status;
+    p.e = epi;
+    switch (pl.bn_idx) {
+        case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);
+        case 1: return tc_launch<32>(st, tw.map, ta.map[1], p, pl.grid, chained);
+        case 2: return tc_launch<64>(st, tw.map, ta.map[2], p, pl.grid, chained);
+        case 3: return tc_launch<128>(st, tw.map, ta.map[3], p, pl.grid, chained);
+        default: return tc_launch<256>(st, tw.map, ta.map[4], p, pl.grid, chained);
     }
-    if (rc) return rc;
-    (*launches)++;
-    if (p.n_splits > 1) {
-        const size_t n = (size_t)n_rows * n_out;
-        splitk_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partial, p.n_splits, p.rows_pad, n_rows, n_out,
-                                                                          Y, ldy, resid);
-        if (cudaGetLastError() != cudaSuccess) return RD_E_CUDA;
-        (*launches)++;
-    }
-    return RD_OK;
 }
 
 }  // namespace rd

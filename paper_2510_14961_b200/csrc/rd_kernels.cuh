@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "rd_common.cuh"
+
 namespace rd {
 
 typedef __nv_bfloat16 bf16;
@@ -81,6 +83,7 @@ __global__ void plan_rows_kernel(const int* __restrict__ n_committed, const int*
                                  const int* __restrict__ done, int B, int Wmax, int* __restrict__ row_pos,
                                  int* __restrict__ row_seq, int* __restrict__ step_first,
                                  int* __restrict__ step_n) {
+    pdl_enter();
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= B * Wmax) return;
     const int b = s / Wmax, j = s % Wmax;
@@ -95,6 +98,7 @@ __global__ void plan_rows_kernel(const int* __restrict__ n_committed, const int*
 // Prefill: n consecutive positions of one sequence.
 __global__ void fill_rows_kernel(int seq, int start, int n, int n_slots, int* __restrict__ row_pos,
                                  int* __restrict__ row_seq) {
+    pdl_enter();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_slots) return;
     row_pos[i] = i < n ? start + i : -1;
@@ -104,13 +108,21 @@ __global__ void fill_rows_kernel(int seq, int start, int n, int n_slots, int* __
 // s_0 ~ N(0, sigma^2 I), keyed by (seed, sequence, position): element j is output j%4 of block
 // j/4; the block's words x0..x3 give two Box-Muller pairs.  Evaluated in double (a few thousand
 // values per new row).  only_fresh: fill rows whose step counter is 0 (rows appended last step).
+// With z_prev the kernel also takes the snapshot z_prev <- z of every active row (Algorithm 2).
 __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                                   const int* __restrict__ row_steps, int only_fresh, int hidden,
-                                  float sigma, uint64_t seed, float* __restrict__ z, size_t ldz) {
+                                  float sigma, uint64_t seed, float* __restrict__ z, size_t ldz,
+                                  float* __restrict__ z_prev) {
+    pdl_enter();
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
-    if (only_fresh && row_steps[r] != 0) return;
+    if (only_fresh && row_steps[r] != 0) {
+        // a row already in flight: only the snapshot z_prev <- z of the step's start is taken
+        if (z_prev)
+            for (int j = threadIdx.x; j < hidden; j += blockDim.x) z_prev[(size_t)r * ldz + j] = z[(size_t)r * ldz + j];
+        return;
+    }
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const int nb = (hidden + 3) / 4;
     for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
@@ -129,7 +141,10 @@ __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __
         }
 #pragma unroll
         for (int a = 0; a < 4; a++)
-            if (blk * 4 + a < hidden) z[(size_t)r * ldz + blk * 4 + a] = out[a];
+            if (blk * 4 + a < hidden) {
+                z[(size_t)r * ldz + blk * 4 + a] = out[a];
+                if (z_prev) z_prev[(size_t)r * ldz + blk * 4 + a] = out[a];
+            }
     }
 }
 
@@ -138,6 +153,7 @@ template <typename T>
 __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                              const int* __restrict__ tokens, int tok_stride, const T* __restrict__ emb,
                              int hidden, float* __restrict__ x) {
+    pdl_enter();
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
@@ -151,6 +167,7 @@ template <typename TO>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, size_t ldx, const float* __restrict__ g,
                                int hidden, float eps, TO* __restrict__ out, size_t ldo,
                                const int* __restrict__ row_pos) {
+    pdl_enter();
     __shared__ float sm[32];
     const int r = blockIdx.x;
     if (row_pos && row_pos[r] < 0) return;
@@ -168,6 +185,7 @@ template <typename T>
 __global__ void concat_kernel(const float* __restrict__ e, size_t lde, const float* __restrict__ z,
                               size_t ldz, int hidden, T* __restrict__ act, size_t lda,
                               const int* __restrict__ row_pos) {
+    pdl_enter();
     const int r = blockIdx.x;
     if (row_pos[r] < 0) return;
     for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
@@ -182,6 +200,7 @@ template <typename T, int RT>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const T* __restrict__ A, size_t lda, const T* __restrict__ W, int K, int n_out,
                  float* __restrict__ Y, size_t ldy, const float* __restrict__ resid, size_t ldr, int n_rows) {
+    pdl_enter();
     constexpr int VEC = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -223,6 +242,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const int* __restr
                                const int* __restrict__ row_seq, const float* __restrict__ cos_t,
                                const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
                                T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride) {
+    pdl_enter();
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
@@ -252,6 +272,7 @@ __global__ void __launch_bounds__(128)
 attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                 const T* __restrict__ Kc, const T* __restrict__ Vc, size_t seq_stride, int hidden,
                 int head_dim, float scale, T* __restrict__ out) {
+    pdl_enter();
     __shared__ float sm_m[4], sm_l[4], sm_o[4][128];
     const int r = blockIdx.x, hd = blockIdx.y;
     const int p = row_pos[r];
@@ -309,14 +330,19 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
     }
 }
 
-// act[r, j] = silu(gu[r, j]) * gu[r, I + j]
+// act[r, j] = silu(gate_j) * up_j.  Plain layout: gu[r] = [gate_0..gate_{I-1} | up_0..up_{I-1}].
+// Interleaved layout (the weight rows were reordered at load for the tensor-core epilogue): groups
+// of 32 = 16 gate features followed by the 16 matching up features.
 template <typename T>
 __global__ void swiglu_kernel(const float* __restrict__ gu, int inner, T* __restrict__ act, size_t lda,
-                              int n_rows) {
+                              int n_rows, int interleaved) {
+    pdl_enter();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)n_rows * inner) return;
     const size_t r = i / inner, j = i % inner;
-    const float g = gu[r * 2 * inner + j], u = gu[r * 2 * inner + inner + j];
+    const size_t gi = interleaved ? (j >> 4) * 32 + (j & 15) : j;
+    const size_t ui = interleaved ? gi + 16 : inner + j;
+    const float g = gu[r * 2 * inner + gi], u = gu[r * 2 * inner + ui];
     act[r * lda + j] = from_f<T>((g / (1.0f + expf(-g))) * u);
 }
 
@@ -327,6 +353,7 @@ __global__ void __launch_bounds__(256)
 sample_kernel(const float* __restrict__ logits, int vocab, const int* __restrict__ row_pos,
               const int* __restrict__ row_seq, float temperature, uint64_t seed, int* __restrict__ draft,
               int* __restrict__ tokens, int tok_stride) {
+    pdl_enter();
     __shared__ float sv[8];
     __shared__ int si[8];
     const int r = blockIdx.x;
@@ -378,6 +405,7 @@ sample_kernel(const float* __restrict__ logits, int vocab, const int* __restrict
 __global__ void __launch_bounds__(256)
 delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int hidden,
              const int* __restrict__ row_pos, float* __restrict__ delta) {
+    pdl_enter();
     __shared__ float sm[32];
     const int r = blockIdx.x;
     if (row_pos[r] < 0) return;
@@ -402,6 +430,7 @@ struct SeqState {
 };
 __global__ void advance_kernel(SeqState st, const float* __restrict__ delta, int B, int Wmax, int window,
                                int inner_iters, float exit_threshold, int cap, int max_new) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B || st.done[b]) return;
     const int f = st.n_committed[b] - 1;
@@ -445,6 +474,18 @@ template <typename T>
 __global__ void convert_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         dst[i] = from_f<T>(src[i]);
+}
+// Gate/up rows reordered for the fused SwiGLU epilogue: destination row (j/16)*32 + j%16 takes gate
+// feature j, row (j/16)*32 + 16 + j%16 takes up feature j.  src = [gate rows | up rows], K columns.
+template <typename T>
+__global__ void interleave_gate_up_kernel(const T* __restrict__ src, T* __restrict__ dst, int inner, int K) {
+    const size_t n = (size_t)2 * inner * K;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t row = i / K, k = i % K;
+        const size_t j = row % inner;
+        const size_t drow = (j >> 4) * 32 + (j & 15) + (row >= (size_t)inner ? 16 : 0);
+        dst[drow * K + k] = src[i];
+    }
 }
 template <typename T>
 __global__ void widen_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {

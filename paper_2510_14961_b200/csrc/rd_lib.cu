@@ -94,6 +94,8 @@ struct rd_model {
     std::vector<LayerW> layers[3];
     TcWeight t_adapter, t_head;
     bool tc_ok = false;
+    bool gu_interleaved = false;   // gate/up rows stored in groups of 16 gate + 16 up (see swiglu_kernel)
+    int n_sms = 148;
 };
 
 static int n_layers_of(const rd_config& c, int blk) { return blk == 0 ? c.n_prelude : blk == 1 ? c.n_core : c.n_coda; }
@@ -123,8 +125,10 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
     const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
     float* stage = nullptr;
     size_t stage_n = 0;
+    void* gu_tmp = nullptr;
     int rc = RD_OK;
     int idx = 0;
+    m->gu_interleaved = c.dtype == RD_BF16 && c.mlp_inner % 16 == 0;
     auto mat = [&](void* dst, size_t n) -> int { return put_tensor(m, dst, t[idx++], n, elem_bytes, &stage, &stage_n); };
     auto gain = [&](float** dst) -> int {
         RD_TRY(m->mem.get(dst, h * sizeof(float)));
@@ -145,8 +149,19 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
                 if ((rc = mat(L.wo, h * h))) break;
                 if ((rc = gain(&L.g2))) break;
                 if ((rc = m->mem.get(&L.wgu, 2 * I * h * es))) break;
-                if ((rc = mat(L.wgu, I * h))) break;
-                if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
+                if (m->gu_interleaved) {
+                    // [gate | up] into a temporary, then rows regrouped 16 gate + 16 up
+                    if (!gu_tmp && (rc = m->mem.get(&gu_tmp, 2 * I * h * es))) break;
+                    if ((rc = mat(gu_tmp, I * h))) break;
+                    if ((rc = mat((char*)gu_tmp + I * h * es, I * h))) break;
+                    interleave_gate_up_kernel<bf16><<<2048, 256>>>((const bf16*)gu_tmp, (bf16*)L.wgu, (int)I, (int)h);
+                    cudaError_t e = cudaGetLastError();
+                    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+                    if (e != cudaSuccess) { rc = cuda_fail(e, "interleave_gate_up_kernel", __LINE__); break; }
+                } else {
+                    if ((rc = mat(L.wgu, I * h))) break;
+                    if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
+                }
                 if ((rc = m->mem.get(&L.wd, h * I * es))) break;
                 if ((rc = mat(L.wd, h * I))) break;
             }
@@ -164,6 +179,7 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
         }
     } while (0);
     if (stage) cudaFree(stage);
+    if (gu_tmp) m->mem.release(gu_tmp);
     if (rc) return rc;
     // Tensor-core path: TMA descriptors over every weight matrix (bf16 only).
     m->tc_ok = false;
@@ -203,6 +219,7 @@ extern "C" int rd_load(const rd_config* cfg, const void* const* tensors, int32_t
     m->cfg = c;
     m->esz = c.dtype == RD_BF16 ? 2 : 4;
     cudaError_t e = cudaGetDevice(&m->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&m->n_sms, cudaDevAttrMultiProcessorCount, m->device);
     if (e != cudaSuccess) { delete m; return cuda_fail(e, "cudaGetDevice", __LINE__); }
     const int rc = load_impl(m, tensors, elem_bytes);
     if (rc) { delete m; return rc; }
@@ -231,8 +248,11 @@ struct rd_session {
     int* status = nullptr;   // device word: non-zero when a bounded wait ran out
     float *x = nullptr, *qkv = nullptr, *gu = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
     float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
-    float* partial = nullptr;   // split-K partial sums of the tensor-core GEMM
-    size_t partial_elems = 0;
+    float* tc_scratch = nullptr;   // partial sums of tiles whose K range is shared between CTAs
+    size_t tc_scratch_elems = 0;
+    int* tc_counters = nullptr;    // per-tile arrival counters (zero between launches)
+    size_t tc_counter_elems = 0;
+    bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
     float *att_o = nullptr, *att_ml = nullptr;   // split-KV partials of the windowed attention
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
@@ -273,12 +293,6 @@ static int bracket_open(rd_session* s, int kind, uint64_t bytes) {
 static void bracket_close(rd_session* s, int idx) {
     if (idx >= 0) cudaEventRecord(s->brackets[idx].b, s->stream);
 }
-
-#define LAUNCHED(s)                  \
-    do {                             \
-        (s)->stats.kernel_launches++; \
-        CU(cudaGetLastError());      \
-    } while (0)
 
 extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp, void* cuda_stream,
                                  rd_session** out) {
@@ -360,8 +374,10 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
             s->attn_path = 1;
         }
         if (m->tc_ok) {
-            s->partial_elems = tc_partial_elems(R, c);
-            if ((rc = s->mem.get(&s->partial, s->partial_elems * sizeof(float)))) break;
+            s->tc_scratch_elems = tc_scratch_elems(R, m->n_sms);
+            if ((rc = s->mem.get(&s->tc_scratch, s->tc_scratch_elems * sizeof(float)))) break;
+            s->tc_counter_elems = tc_counter_elems(R, std::max(std::max(3 * c.hidden, 2 * c.mlp_inner), c.vocab));
+            if ((rc = s->mem.get(&s->tc_counters, s->tc_counter_elems * sizeof(int)))) break;
             bool ok = tc_make_act(&s->t_act_h, s->act_h, (int)Ra, c.hidden) == RD_OK;
             ok &= tc_make_act(&s->t_act_2h, s->act_2h, (int)Ra, 2 * c.hidden) == RD_OK;
             ok &= tc_make_act(&s->t_act_i, s->act_i, (int)Ra, c.mlp_inner) == RD_OK;
@@ -383,37 +399,63 @@ extern "C" void rd_session_destroy(rd_session* s) {
 }
 extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
     if (!s || (path != 0 && path != 1)) return RD_E_INVALID_ARG;
-    if (path == 1 && !(s->m->tc_ok && s->partial)) return RD_E_STATE;
+    if (path == 1 && !(s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
     s->gemm_path = path;
+    return RD_OK;
+}
+
+extern "C" int rd_set_launch_chaining(rd_session* s, int32_t on) {
+    if (!s || (on != 0 && on != 1)) return RD_E_INVALID_ARG;
+    s->chained = on != 0;
     return RD_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
 // The schedule (templated on the storage type T of weights / KV / GEMM inputs)
 // ---------------------------------------------------------------------------------------------
+// Every kernel of a step is a link of one programmatic-dependent-launch chain (rd_common.cuh).
+#define LAUNCH(s, kern, grid, block, smem, ...)                                                   \
+    do {                                                                                          \
+        cudaError_t e_ = launch_chained(kern, dim3(grid), dim3(block), smem, (s)->stream, (s)->chained, __VA_ARGS__); \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #kern, __LINE__);                             \
+        (s)->stats.kernel_launches++;                                                             \
+    } while (0)
+
 template <typename T> struct Eng {
-    // Y[r, o] = sum_k A[r, k] W[o, k] (+ resid).  `ta`/`tw` are the operands' TMA descriptors for
+    static bool tc_usable(const rd_session* s, const TcAct* ta, const TcWeight* tw) {
+        return sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid;
+    }
+    static int tc_run(rd_session* s, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
+                      const TcEpilogue& epi) {
+        const int rc = tc_gemm(s->stream, ta, tw, K, n_out, n_rows, epi, s->tc_scratch, s->tc_scratch_elems,
+                               s->tc_counters, s->tc_counter_elems, s->m->n_sms, s->status, s->chained);
+        if (rc == RD_OK) { s->stats.tc_gemm_launches++; s->stats.kernel_launches++; }
+        else if (rc == RD_E_CUDA) return cuda_fail(cudaGetLastError(), "tensor-core GEMM launch", __LINE__);
+        return rc;
+    }
+
+    // Y[r, o] = sum_k A[r, k] W[o, k] (+ resid[r, o]).  `ta`/`tw` are the operands' TMA descriptors for
     // the tensor-core path (bf16 only).
     static int gemm(rd_session* s, const T* A, size_t lda, const TcAct* ta, const T* W, const TcWeight* tw, int K,
                     int n_out, float* Y, size_t ldy, const float* resid, int n_rows) {
         const int br = bracket_open(s, 0, (uint64_t)n_out * K * sizeof(T));
-        if (sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid) {
-            const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, Y, ldy, resid, n_rows, s->partial,
-                                   s->partial_elems, s->status, &s->stats.kernel_launches);
-            if (rc == RD_OK) { s->stats.tc_gemm_launches++; bracket_close(s, br); return RD_OK; }
+        if (tc_usable(s, ta, tw)) {
+            TcEpilogue e = {};
+            e.mode = TC_EPI_STORE; e.Y = Y; e.ldy = ldy; e.resid = resid; e.ldr = ldy;
+            const int rc = tc_run(s, *ta, *tw, K, n_out, n_rows, e);
+            if (rc == RD_OK) { bracket_close(s, br); return RD_OK; }
             if (rc != RD_E_INVALID_ARG) return rc;   // INVALID_ARG: shape not taken, fall through
         }
         const int warps = 8;
         dim3 grid((n_out + warps - 1) / warps, 1);
         if (n_rows == 1) {
-            gemm_simt_kernel<T, 1><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 1>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
         } else if (n_rows <= 4) {
-            gemm_simt_kernel<T, 4><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 4>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
         } else {
             grid.y = (n_rows + 7) / 8;
-            gemm_simt_kernel<T, 8><<<grid, warps * 32, 0, s->stream>>>(A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 8>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
         }
-        LAUNCHED(s);
         bracket_close(s, br);
         return RD_OK;
     }
@@ -429,16 +471,14 @@ template <typename T> struct Eng {
         const rd_config& c = s->m->cfg;
         const int groups = (n_rows + s->grp_rows - 1) / s->grp_rows;
         const int tiles = std::max(1, (s->ctx_max + ATT_KT - 1) / ATT_KT);
-        int ns = (2 * 148 + groups * c.n_heads - 1) / (groups * c.n_heads);
+        int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
         ns = std::max(1, std::min(std::min(ns, 8), tiles));
         const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
-        attn_window_kernel<D><<<dim3(c.n_heads, groups, ns), 128, AttCfg<D>::SMEM, s->stream>>>(
-            (const bf16*)s->q_t, s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden,
-            scale_log2, ns, s->att_o, s->att_ml);
-        LAUNCHED(s);
-        attn_combine_kernel<D><<<dim3(n_rows, c.n_heads), D, 0, s->stream>>>(s->att_o, s->att_ml, ns, s->row_pos,
-                                                                              c.hidden, (bf16*)s->act_h);
-        LAUNCHED(s);
+        LAUNCH(s, attn_window_kernel<D>, dim3(c.n_heads, groups, ns), 128, AttCfg<D>::SMEM, (const bf16*)s->q_t,
+               s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden, scale_log2, ns, s->att_o,
+               s->att_ml);
+        LAUNCH(s, attn_combine_kernel<D>, dim3(n_rows, c.n_heads), D, 0, s->att_o, s->att_ml, ns, s->row_pos, c.hidden,
+               (bf16*)s->act_h);
         return RD_OK;
     }
     static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {
@@ -450,20 +490,35 @@ template <typename T> struct Eng {
         }
     }
 
-    // One transformer layer over the rows of the current row table, in place on x.
-    static int layer(rd_session* s, int blk, int l, float* x, int n_rows) {
+    // One transformer layer over the rows of the current row table: reads x_in, leaves the
+    // mid-layer residual in s->x, writes x_out (x_in, x_out may both be s->x).
+    static int layer(rd_session* s, int blk, int l, const float* x_in, float* x_out, int n_rows) {
         const rd_config& c = s->m->cfg;
         const LayerW& L = s->m->layers[blk][l];
         const int h = c.hidden, I = c.mlp_inner;
         const size_t layer_off = (size_t)l * s->sc.batch * s->seq_stride;
         T* Kc = (T*)s->Kc[blk] + layer_off;
         T* Vc = (T*)s->Vc[blk] + layer_off;
-        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g1, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
-        LAUNCHED(s);
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, s->qkv, 3 * h, nullptr, n_rows));
-        rope_kv_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->qkv, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h,
-                                                          c.head_dim, (T*)s->q_t, Kc, Vc, s->seq_stride);
-        LAUNCHED(s);
+        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, x_in, (size_t)h, L.g1, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
+        // q, k, v: on the tensor-core path the rotary embedding and the cache write are the GEMM's epilogue
+        bool qkv_done = false;
+        if constexpr (sizeof(T) == 2) {
+            if (tc_usable(s, &s->t_act_h, &L.t_qkv)) {
+                const int br = bracket_open(s, 0, (uint64_t)3 * h * h * sizeof(T));
+                TcEpilogue e = {};
+                e.mode = TC_EPI_QKV; e.q_t = (bf16*)s->q_t; e.Kc = (bf16*)Kc; e.Vc = (bf16*)Vc; e.seq_stride = s->seq_stride;
+                e.hidden = h; e.head_dim = c.head_dim; e.row_pos = s->row_pos; e.row_seq = s->row_seq;
+                e.cos_t = s->cos_t; e.sin_t = s->sin_t;
+                const int rc = tc_run(s, s->t_act_h, L.t_qkv, h, 3 * h, n_rows, e);
+                if (rc == RD_OK) { bracket_close(s, br); qkv_done = true; }
+                else if (rc != RD_E_INVALID_ARG) return rc;
+            }
+        }
+        if (!qkv_done) {
+            RD_TRY(gemm(s, (T*)s->act_h, h, nullptr, (T*)L.wqkv, nullptr, h, 3 * h, s->qkv, 3 * h, nullptr, n_rows));
+            LAUNCH(s, rope_kv_kernel<T>, n_rows, 256, 0, s->qkv, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+                   (T*)s->q_t, Kc, Vc, s->seq_stride);
+        }
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
         if constexpr (sizeof(T) == 2) {
@@ -473,30 +528,41 @@ template <typename T> struct Eng {
             }
         }
         if (!windowed) {
-            attn_row_kernel<T><<<dim3(n_rows, c.n_heads), 128, 0, s->stream>>>(
-                (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc, s->seq_stride, h, c.head_dim,
-                (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
-            LAUNCHED(s);
+            LAUNCH(s, attn_row_kernel<T>, dim3(n_rows, c.n_heads), 128, 0, (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc,
+                   s->seq_stride, h, c.head_dim, (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
         }
         bracket_close(s, br);
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, x, h, x, n_rows));
-        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(x, h, L.g2, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
-        LAUNCHED(s);
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, s->gu, 2 * I, nullptr, n_rows));
-        const size_t n_el = (size_t)n_rows * I;
-        swiglu_kernel<T><<<(unsigned)((n_el + 255) / 256), 256, 0, s->stream>>>(s->gu, I, (T*)s->act_i, I, n_rows);
-        LAUNCHED(s);
-        RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, x, h, x, n_rows));
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, s->x, h, x_in, n_rows));
+        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, s->x, (size_t)h, L.g2, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
+        // gate/up: with interleaved weight rows SwiGLU is the GEMM's epilogue
+        bool mlp_done = false;
+        if constexpr (sizeof(T) == 2) {
+            if (s->m->gu_interleaved && tc_usable(s, &s->t_act_h, &L.t_gu)) {
+                const int br2 = bracket_open(s, 0, (uint64_t)2 * I * h * sizeof(T));
+                TcEpilogue e = {};
+                e.mode = TC_EPI_SWIGLU; e.act = (bf16*)s->act_i; e.lda = I; e.inner = I;
+                const int rc = tc_run(s, s->t_act_h, L.t_gu, h, 2 * I, n_rows, e);
+                if (rc == RD_OK) { bracket_close(s, br2); mlp_done = true; }
+                else if (rc != RD_E_INVALID_ARG) return rc;
+            }
+        }
+        if (!mlp_done) {
+            RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, s->gu, 2 * I, nullptr, n_rows));
+            const size_t n_el = (size_t)n_rows * I;
+            LAUNCH(s, swiglu_kernel<T>, (unsigned)((n_el + 255) / 256), 256, 0, s->gu, I, (T*)s->act_i, (size_t)I, n_rows,
+                   s->m->gu_interleaved ? 1 : 0);
+        }
+        RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, x_out, h, s->x, n_rows));
         return RD_OK;
     }
 
-    // e = P(tokens of the rows): embedding + prelude layers; result left in s->x.
-    static int prelude(rd_session* s, int n_rows) {
+    // e_out = P(tokens of the rows): embedding + prelude layers.
+    static int prelude(rd_session* s, int n_rows, float* e_out) {
         const rd_config& c = s->m->cfg;
-        embed_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->row_pos, s->row_seq, s->tokens, s->tok_stride,
-                                                        (const T*)s->m->emb, c.hidden, s->x);
-        LAUNCHED(s);
-        for (int l = 0; l < c.n_prelude; l++) RD_TRY(layer(s, 0, l, s->x, n_rows));
+        float* x0 = c.n_prelude > 0 ? s->x : e_out;
+        LAUNCH(s, embed_kernel<T>, n_rows, 256, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride, (const T*)s->m->emb,
+               c.hidden, x0);
+        for (int l = 0; l < c.n_prelude; l++) RD_TRY(layer(s, 0, l, s->x, l == c.n_prelude - 1 ? e_out : s->x, n_rows));
         return RD_OK;
     }
 
@@ -504,13 +570,11 @@ template <typename T> struct Eng {
     static int core(rd_session* s, const float* e, const float* z_in, float* z_out, int n_rows) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
-        concat_kernel<T><<<n_rows, 256, 0, s->stream>>>(e, h, z_in, h, h, (T*)s->act_2h, 2 * h, s->row_pos);
-        LAUNCHED(s);
+        LAUNCH(s, concat_kernel<T>, n_rows, 256, 0, e, (size_t)h, z_in, (size_t)h, h, (T*)s->act_2h, (size_t)2 * h, s->row_pos);
         RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, s->x, h,
                     nullptr, n_rows));
-        for (int l = 0; l < c.n_core; l++) RD_TRY(layer(s, 1, l, s->x, n_rows));
-        rmsnorm_kernel<float><<<n_rows, 256, 0, s->stream>>>(s->x, h, s->m->g_core, h, c.norm_eps, z_out, h, s->row_pos);
-        LAUNCHED(s);
+        for (int l = 0; l < c.n_core; l++) RD_TRY(layer(s, 1, l, s->x, s->x, n_rows));
+        LAUNCH(s, rmsnorm_kernel<float>, n_rows, 256, 0, s->x, (size_t)h, s->m->g_core, h, c.norm_eps, z_out, (size_t)h, s->row_pos);
         return RD_OK;
     }
 
@@ -518,16 +582,14 @@ template <typename T> struct Eng {
     static int coda(rd_session* s, const float* z, int n_rows, bool head) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
-        CU(cudaMemcpyAsync(s->x, z, (size_t)n_rows * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
-        for (int l = 0; l < c.n_coda; l++) RD_TRY(layer(s, 2, l, s->x, n_rows));
+        for (int l = 0; l < c.n_coda; l++) RD_TRY(layer(s, 2, l, l == 0 ? z : s->x, s->x, n_rows));
         if (!head) return RD_OK;
-        rmsnorm_kernel<T><<<n_rows, 256, 0, s->stream>>>(s->x, h, s->m->g_final, h, c.norm_eps, (T*)s->act_h, h, s->row_pos);
-        LAUNCHED(s);
+        const float* xf = c.n_coda > 0 ? s->x : z;
+        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, xf, (size_t)h, s->m->g_final, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, s->logits, c.vocab,
                     nullptr, n_rows));
-        sample_kernel<<<n_rows, 256, 0, s->stream>>>(s->logits, c.vocab, s->row_pos, s->row_seq, s->sc.temperature,
-                                                     s->sc.seed, s->draft, s->tokens, s->tok_stride);
-        LAUNCHED(s);
+        LAUNCH(s, sample_kernel, n_rows, 256, 0, s->logits, c.vocab, s->row_pos, s->row_seq, s->sc.temperature, s->sc.seed,
+               s->draft, s->tokens, s->tok_stride);
         return RD_OK;
     }
 
@@ -546,30 +608,51 @@ template <typename T> struct Eng {
                 s->ctx_total += ctx;
                 s->ctx_max = std::max(s->ctx_max, ctx);
             }
-        plan_rows_kernel<<<(n + 127) / 128, 128, 0, s->stream>>>(s->n_committed, s->win_len, s->done, B,
-                                                                 s->sc.max_window, s->row_pos, s->row_seq,
-                                                                 s->step_first, s->step_n);
-        LAUNCHED(s);
-        init_state_kernel<<<n, 128, 0, s->stream>>>(s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma,
-                                                    s->sc.seed, s->z, h);
-        LAUNCHED(s);
-        CU(cudaMemcpyAsync(s->z_prev, s->z, (size_t)n * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
-        RD_TRY(prelude(s, n));
-        CU(cudaMemcpyAsync(s->e, s->x, (size_t)n * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
+        LAUNCH(s, plan_rows_kernel, (n + 127) / 128, 128, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window,
+               s->row_pos, s->row_seq, s->step_first, s->step_n);
+        // s_0 for the rows appended by the previous step, and the snapshot z_prev <- z
+        LAUNCH(s, init_state_kernel, n, 128, 0, s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma, s->sc.seed, s->z,
+               (size_t)h, s->z_prev);
+        RD_TRY(prelude(s, n, s->e));
         for (int j = 0; j < inner; j++) RD_TRY(core(s, s->e, s->z, s->z, n));
         RD_TRY(coda(s, s->z, n, true));
-        delta_kernel<<<n, 256, 0, s->stream>>>(s->z, s->z_prev, h, s->row_pos, s->delta);
-        LAUNCHED(s);
+        LAUNCH(s, delta_kernel, n, 256, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
         SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
-        advance_kernel<<<(B + 63) / 64, 64, 0, s->stream>>>(st, s->delta, B, s->sc.max_window, window, inner, eps,
-                                                            s->sc.max_iters_per_pos, s->sc.max_new_tokens);
-        LAUNCHED(s);
+        LAUNCH(s, advance_kernel, (B + 63) / 64, 64, 0, st, s->delta, B, s->sc.max_window, window, inner, eps,
+               s->sc.max_iters_per_pos, s->sc.max_new_tokens);
+        return RD_OK;
+    }
+
+    static int prefill_passes(rd_session* s, int seq, int n, int r, float* e_all, float* s_all) {
+        const rd_config& c = s->m->cfg;
+        const int h = c.hidden;
+        for (int pass = 0; pass < r + 2; pass++) {
+            // pass 0: P and s_0 for every chunk; passes 1..r: one simultaneous application of R;
+            // pass r+1: coda layers (fills the coda cache; no head).
+            for (int c0 = 0; c0 < n; c0 += s->R) {
+                const int nr = std::min(s->R, n - c0);
+                s->grp_rows = ATT_QMAX;
+                s->ctx_max = c0 + nr;
+                s->ctx_total = c0 + nr;
+                LAUNCH(s, fill_rows_kernel, (s->R + 127) / 128, 128, 0, seq, c0, nr, s->R, s->row_pos, s->row_seq);
+                float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
+                float* zc = s_all + (size_t)c0 * h;
+                if (pass == 0) {
+                    RD_TRY(prelude(s, nr, ec));
+                    LAUNCH(s, init_state_kernel, nr, 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
+                           s->sc.seed, zc, (size_t)h, (float*)nullptr);
+                } else if (pass <= r) {
+                    RD_TRY(core(s, ec, zc, zc, nr));
+                } else {
+                    RD_TRY(coda(s, zc, nr, false));
+                }
+            }
+        }
         return RD_OK;
     }
 
     static int prefill(rd_session* s, int seq, const int32_t* prompt, int L, int r) {
-        const rd_config& c = s->m->cfg;
-        const int h = c.hidden;
+        const int h = s->m->cfg.hidden;
         CU(cudaStreamSynchronize(s->stream));
         CU(cudaMemcpy(s->tokens + (size_t)seq * s->tok_stride, prompt, (size_t)L * sizeof(int), cudaMemcpyHostToDevice));
         const int n = L - 1;   // rows 0..L-2 are prefilled; L-1 is the first in-flight row
@@ -578,37 +661,14 @@ template <typename T> struct Eng {
         if (n > 0) {
             RD_TRY(s->mem.get(&e_all, (size_t)n * h * sizeof(float)));
             rc = s->mem.get(&s_all, (size_t)n * h * sizeof(float));
-        }
-        for (int pass = 0; pass < r + 2 && !rc && n > 0; pass++) {
-            // pass 0: P and s_0 for every chunk; passes 1..r: one simultaneous application of R;
-            // pass r+1: coda layers (fills the coda cache; no head).
-            for (int c0 = 0; c0 < n && !rc; c0 += s->R) {
-                const int nr = std::min(s->R, n - c0);
-                s->grp_rows = ATT_QMAX;
-                s->ctx_max = c0 + nr;
-                s->ctx_total = c0 + nr;
-                fill_rows_kernel<<<(s->R + 127) / 128, 128, 0, s->stream>>>(seq, c0, nr, s->R, s->row_pos, s->row_seq);
-                s->stats.kernel_launches++;
-                float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
-                float* zc = s_all + (size_t)c0 * h;
-                if (pass == 0) {
-                    rc = prelude(s, nr);
-                    if (rc) break;
-                    cudaMemcpyAsync(ec, s->x, (size_t)nr * h * sizeof(float), cudaMemcpyDeviceToDevice, s->stream);
-                    init_state_kernel<<<nr, 128, 0, s->stream>>>(s->row_pos, s->row_seq, s->row_steps, 0, h,
-                                                                 c.init_sigma, s->sc.seed, zc, h);
-                    s->stats.kernel_launches++;
-                } else if (pass <= r) {
-                    rc = core(s, ec, zc, zc, nr);
-                } else {
-                    rc = coda(s, zc, nr, false);
-                }
-            }
+            if (!rc) rc = prefill_passes(s, seq, n, r, e_all, s_all);
         }
         if (!rc) {
             cudaError_t e = cudaStreamSynchronize(s->stream);
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess) rc = cuda_fail(e, "prefill", __LINE__);
+        } else {
+            cudaStreamSynchronize(s->stream);
         }
         if (e_all) s->mem.release(e_all);
         if (s_all) s->mem.release(s_all);
