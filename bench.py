@@ -146,7 +146,9 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    wl = WORKLOADS[args.workload]
+    wl = dict(WORKLOADS[args.workload])
+    if args.prefill_r > 0:
+        wl["prefill_r"] = args.prefill_r
     shape, B, L, N, W = wl["shape"], wl["batch"], wl["prompt"], wl["gen"], wl["window"]
     esz = 2 if wl["bf16"] else 4
     peaks = load_peaks()
@@ -434,6 +436,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--ar-tokens", type=int, default=24)
+    ap.add_argument("--prefill-r", type=int, default=0, help="override the workload's prefill recurrence (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

@@ -48,8 +48,8 @@ enum {
 typedef struct rd_model rd_model;     /* opaque: device weights                          */
 typedef struct rd_session rd_session; /* opaque: KV caches, latents, tokens, wavefront   */
 
-/* Model shape.  hidden must equal n_heads * head_dim; hidden and mlp_inner must be multiples of
- * 8, head_dim even and <= 128.  dtype selects the storage type of weights, KV cache and GEMM
+/* Model shape.  hidden must equal n_heads * head_dim and be at most 12288; hidden and mlp_inner must
+ * be multiples of 8, head_dim even and <= 128.  dtype selects the storage type of weights, KV cache and GEMM
  * inputs (accumulation, residual stream, latents, softmax and logits are always float32). */
 typedef struct {
     int32_t hidden, n_heads, head_dim, mlp_inner;

@@ -9,27 +9,25 @@
 // (128 lanes x BN columns, fp32, two buffers).
 //
 // Persistent stream-K schedule: the (feature tile, row tile, k-block) units are numbered tile by
-// tile and cut into one contiguous share per CTA (one CTA per SM), so every SM streams the same
-// number of weight bytes through one long-lived ring whatever n_out is.  A share is a list of
-// segments (tile, k-block range):
+// tile and cut into one contiguous share per CTA (two CTAs per SM while the row tile is at most
+// 64 wide), so every SM streams the same number of weight bytes through long-lived rings whatever
+// n_out is.  A share is a list of segments (tile, k-block range):
 //   warp 0 / lane 0   TMA producer: fills a ring of STAGES {A,B} stages, mbarrier complete_tx
 //   warp 1 / lane 0   issues tcgen05.mma (4 per stage, K = 16 each); tcgen05.commit frees the stage
 //                     and, at the end of a segment, publishes the accumulator buffer
-//   warps 2-5         epilogue: tcgen05.ld of their 32 TMEM lanes; the next segment's MMAs run
-//                     meanwhile in the other accumulator buffer
-// A segment that covers the whole K range is finished from TMEM.  Otherwise its fp32 partial goes
-// to a scratch slot and a per-tile counter is bumped; the CTA that brings the counter to the
-// number of segments of the tile adds all partials IN K ORDER and finishes the tile.  No float
-// atomics and no order that depends on timing: results are bit-reproducible.  Nobody waits for
-// another CTA.
-//
-// Finishing a tile applies the fused epilogue: store (+ residual); SwiGLU on interleaved gate/up
-// features -> bf16; rotary embedding on q,k -> q buffer and the K/V cache entries of the rows.
+//   warps 2-5         tcgen05.ld of their 32 TMEM lanes, coalesced stores; the next segment's MMAs
+//                     run meanwhile in the other accumulator buffer
+// The kernel does not finish the sums.  Each segment's fp32 partial sums go to their own slot of a
+// scratch buffer (rd_partial.cuh), and the kernel that consumes the GEMM's result (normalisation,
+// rotary embedding + cache write, SwiGLU, sampling) adds a tile's slots in ascending k order while
+// it reads.  So there are no float atomics, no fences, no counters, nobody waits for another CTA,
+// and results are bit-reproducible.  (Measured on B200: finishing split tiles inside the kernel,
+// last arriver adds, cost 8-11 us per launch; the kernels here run 15-110 us.)
 //
 // Programmatic dependent launch: the kernel lets its successor start at once, and itself starts
-// while its predecessor still runs: it sets up, prefetches the first weight stages (weights do not
-// depend on earlier kernels), and only then waits for the predecessor before touching activations
-// or outputs.
+// while its predecessor still runs: it sets up, requests its first ring of weight tiles (weights
+// do not depend on earlier kernels), and only then waits for the predecessor before touching
+// activations or the scratch buffer.
 //
 // Every wait on an mbarrier is bounded; on time-out the kernel raises a status word, drains the
 // copies it issued, frees its TMEM and returns.
@@ -43,6 +41,7 @@
 
 #include "../../include/rd.h"
 #include "rd_common.cuh"
+#include "rd_partial.cuh"
 
 namespace rd {
 
@@ -50,8 +49,6 @@ constexpr int TC_BM = 128;       // output features per tile (UMMA M)
 constexpr int TC_BK = 64;        // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
-
-enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_QKV = 2 };
 
 struct TcWeight {
     CUtensorMap map;
@@ -191,97 +188,34 @@ __host__ __device__ constexpr uint32_t umma_idesc(int bn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+#ifndef RD_TC_RING_KB
+#define RD_TC_RING_KB 100
+#endif
+constexpr int TC_CTAS_PER_SM = 2;   // while BN <= 64
+
 template <int BN> struct TcCfg {
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;                 // 16 KB
     static constexpr int B_BYTES = BN * TC_BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // about 200 KB of ring per CTA (one CTA per SM): enough bytes in flight to cover HBM latency at
-    // full bandwidth, and a CTA that starts early under programmatic dependent launch prefetches
-    // that much of its weights while the kernels before it finish
-    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 12 ? 12 : (200 * 1024) / STAGE_BYTES;
+    // Two CTAs per SM with about 100 KB of ring each (measured: two independent producer / MMA
+    // pipelines per SM stream at the HBM peak, one with a ring twice as deep at 80 % of it).
+    // Row tiles wider than 64 take the whole SM.
+    static constexpr int RING_KB = BN <= 64 ? RD_TC_RING_KB : 200;
+    static constexpr int STAGES = (RING_KB * 1024) / STAGE_BYTES > 12 ? 12 : (RING_KB * 1024) / STAGE_BYTES;
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;                // columns of one accumulator buffer
     static constexpr int TMEM_COLS = 2 * ACC_COLS;                    // power of two, 64..512
 };
 
-// What finishing a tile does with acc[r, o].
-struct TcEpilogue {
-    int mode;
-    // TC_EPI_STORE: Y[r, o] = acc (+ resid[r, o])
-    float* Y; size_t ldy; const float* resid; size_t ldr;
-    // TC_EPI_SWIGLU: features come in groups of 32 = 16 gate, then the 16 matching up features;
-    // act[r, j] = silu(gate_j) * up_j, j < inner
-    __nv_bfloat16* act; size_t lda; int inner;
-    // TC_EPI_QKV: o in [0, 3 hidden) = q | k | v.  Rotary embedding on adjacent pairs of q and k with
-    // the row's position; q -> q_t[r], k and v -> the row's own cache entry.
-    __nv_bfloat16 *q_t, *Kc, *Vc; size_t seq_stride; int hidden, head_dim;
-    const int *row_pos, *row_seq; const float *cos_t, *sin_t;
-};
-
 struct TcParams {
-    int K, n_out, n_rows;
     int kb;                    // k-blocks per tile
-    int n_tiles_m, n_tiles_n;
+    int n_tiles_m;
     long long units;           // n_tiles_m * n_tiles_n * kb
     int per;                   // units per CTA
-    float* scratch;            // [2 * gridDim.x][BN][128] partial sums
-    int* counters;             // [tiles] arrivals of partial segments; zero between launches
+    int max_seg;               // scratch slots per CTA
+    float* scratch;            // [gridDim.x * max_seg][BN][128] partial sums
     int* status;
-    TcEpilogue e;
 };
-
-// Finish 16 rows (columns c0..c0+15 of the accumulator) of this thread's output feature.
-template <int BN>
-__device__ __forceinline__ void tc_finish_chunk(const TcParams& p, int m0, int n0, int c0, int quad, int lane, const float* v) {
-    const TcEpilogue& e = p.e;
-    const int f = quad * 32 + lane;
-    const int m = m0 + f;
-    if (e.mode == TC_EPI_STORE) {
-        if (m < p.n_out) {
-#pragma unroll
-            for (int j = 0; j < 16; j++) {
-                const int r = n0 + c0 + j;
-                if (r < p.n_rows) e.Y[(size_t)r * e.ldy + m] = e.resid ? e.resid[(size_t)r * e.ldr + m] + v[j] : v[j];
-            }
-        }
-    } else if (e.mode == TC_EPI_SWIGLU) {
-        const int jf = (m0 >> 1) + quad * 16 + (lane & 15);
-#pragma unroll
-        for (int j = 0; j < 16; j++) {
-            const float up = __shfl_xor_sync(0xffffffffu, v[j], 16);
-            const int r = n0 + c0 + j;
-            if (lane < 16 && jf < e.inner && r < p.n_rows) {
-                const float g = v[j];
-                e.act[(size_t)r * e.lda + jf] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * up);
-            }
-        }
-    } else {
-        const int sec = m / e.hidden, mm = m - sec * e.hidden;
-        const int half = e.head_dim >> 1;
-        const int i = (mm % e.head_dim) >> 1;
-        const bool odd = (m & 1) != 0;
-#pragma unroll
-        for (int j = 0; j < 16; j++) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[j], 1);
-            const int r = n0 + c0 + j;
-            if (m >= p.n_out || r >= p.n_rows) continue;
-            const int pos = e.row_pos[r];
-            if (pos < 0) continue;
-            float out = v[j];
-            if (sec < 2) {
-                const float c = e.cos_t[(size_t)pos * half + i], s = e.sin_t[(size_t)pos * half + i];
-                out = odd ? other * s + v[j] * c : v[j] * c - other * s;
-            }
-            const __nv_bfloat16 o16 = __float2bfloat16_rn(out);
-            if (sec == 0) {
-                e.q_t[(size_t)r * e.hidden + mm] = o16;
-            } else {
-                __nv_bfloat16* dst = (sec == 1 ? e.Kc : e.Vc) + (size_t)e.row_seq[r] * e.seq_stride + (size_t)pos * e.hidden;
-                dst[mm] = o16;
-            }
-        }
-    }
-}
 
 template <int BN>
 __global__ void __launch_bounds__(TC_THREADS)
@@ -293,10 +227,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     uint64_t* empty = full + C::STAGES;
     uint64_t* acc_full = empty + C::STAGES;     // [2]
     uint64_t* acc_empty = acc_full + 2;         // [2]
-    uint64_t* epi_bar = acc_empty + 2;          // the 128 epilogue threads meet here (bounded waits)
-    uint32_t* tmem_slot = (uint32_t*)(epi_bar + 1);
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    volatile uint32_t* last_flag = tmem_slot + 2;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long u0 = (long long)blockIdx.x * p.per;
@@ -308,7 +240,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
-        mbar_init(epi_bar, 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -391,80 +322,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (!ok) *abort_flag = 1;
             }
         } else {
-            // ---- epilogue warps 2..5: TMEM lane quadrant = warp % 4 ----
-            const int quad = warp & 3;
-            const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+            // ---- warps 2..5 move finished segments from TMEM to their scratch slot ----
+            const int quad = warp & 3;                    // TMEM lane quadrant a warp may read
             int i = 0, seg = 0;
-            uint32_t epi_phase = 0;
             bool ok = true;
-            // all 128 epilogue threads arrive, then wait for the phase: false if someone never came
-            auto epi_sync = [&]() -> bool {
-                mbar_arrive(epi_bar);
-                const bool done = mbar_wait(epi_bar, epi_phase & 1);
-                epi_phase++;
-                return done;
-            };
             while (i < n_units && ok) {
                 const long long u = u0 + i;
-                const int tile = (int)(u / p.kb), ka = (int)(u % p.kb);
+                const int ka = (int)(u % p.kb);
                 const int len = min(p.kb - ka, n_units - i);
                 const int buf = seg & 1;
-                const int m0 = (tile % p.n_tiles_m) * TC_BM, n0 = (tile / p.n_tiles_m) * BN;
-                const bool whole = (ka == 0 && len == p.kb);
                 if (*abort_flag || !mbar_wait(&acc_full[buf], (seg >> 1) & 1)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_COLS);
-                // first segment of the share -> slot 2g, a later partial one (the last) -> 2g + 1
-                float* slot = p.scratch + ((size_t)blockIdx.x * 2 + (i == 0 ? 0 : 1)) * (size_t)(BN * TC_BM);
+                // the share's seg-th segment (= seg-th tile it touches) -> slot blockIdx.x * max_seg + seg
+                float* slot = p.scratch + ((size_t)blockIdx.x * p.max_seg + seg) * (size_t)(BN * TC_BM) + quad * 32 + lane;
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 16) {
                     uint32_t raw[16];
                     tmem_ld16(t + (uint32_t)c, raw);
-                    float v[16];
 #pragma unroll
-                    for (int j = 0; j < 16; j++) v[j] = __uint_as_float(raw[j]);
-                    if (whole) {
-                        tc_finish_chunk<BN>(p, m0, n0, c, quad, lane, v);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; j++) slot[(size_t)(c + j) * TC_BM + quad * 32 + lane] = v[j];
-                    }
+                    for (int j = 0; j < 16; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);     // accumulator buffer may be overwritten
-                if (!whole) {
-                    // publish the partial; the CTA that completes the tile's count finishes it
-                    const long long t_lo = (long long)tile * p.kb;
-                    const int g_lo = (int)(t_lo / p.per), g_hi = (int)((t_lo + p.kb - 1) / p.per);
-                    __threadfence();
-                    if (!epi_sync()) { ok = false; break; }
-                    if (et == 0) {
-                        const int old = atomicAdd(&p.counters[tile], 1);
-                        const bool last = old == g_hi - g_lo;
-                        if (last) p.counters[tile] = 0;          // ready for the next launch
-                        *last_flag = last ? 1u : 0u;
-                    }
-                    if (!epi_sync()) { ok = false; break; }
-                    if (*last_flag) {
-                        __threadfence();
-#pragma unroll 1
-                        for (int c = 0; c < BN; c += 16) {
-                            float v[16];
-#pragma unroll
-                            for (int j = 0; j < 16; j++) v[j] = 0.f;
-                            for (int g = g_lo; g <= g_hi; g++) {          // ascending k
-                                const int first_tile = (int)(((long long)g * p.per) / p.kb);
-                                const float* sl = p.scratch + ((size_t)g * 2 + (first_tile == tile ? 0 : 1)) * (size_t)(BN * TC_BM);
-#pragma unroll
-                                for (int j = 0; j < 16; j++) v[j] += __ldcg(sl + (size_t)(c + j) * TC_BM + quad * 32 + lane);
-                            }
-                            tc_finish_chunk<BN>(p, m0, n0, c, quad, lane, v);
-                        }
-                    }
-                    // (last_flag is next written after the next segment's first meeting, which every
-                    // thread reaches only after it has read the flag here)
-                }
                 i += len;
                 seg++;
             }
@@ -483,14 +364,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 static inline int tc_pick_bn(int n_rows) { return n_rows <= 16 ? 0 : n_rows <= 32 ? 1 : n_rows <= 64 ? 2 : n_rows <= 128 ? 3 : 4; }
 
 struct TcPlan {
-    int bn_idx, bn, kb, n_tiles_m, n_tiles_n, per, grid;
+    int bn_idx, bn, kb, n_tiles_m, n_tiles_n, per, grid, max_seg;
     long long units;
+    size_t scratch_elems;
 };
-// One CTA per SM; every CTA gets `per` consecutive units (the last ones possibly fewer).
+// Every CTA gets `per` consecutive units (the last ones possibly fewer).
 static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms) {
     TcPlan pl;
     pl.bn_idx = tc_pick_bn(n_rows);
     pl.bn = 16 << pl.bn_idx;
+    if (pl.bn <= 64) n_sms *= TC_CTAS_PER_SM;
     pl.kb = (K + TC_BK - 1) / TC_BK;
     pl.n_tiles_m = (n_out + TC_BM - 1) / TC_BM;
     pl.n_tiles_n = (n_rows + pl.bn - 1) / pl.bn;
@@ -498,16 +381,9 @@ static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms) {
     const long long g = std::min<long long>(n_sms, pl.units);
     pl.per = (int)((pl.units + g - 1) / g);
     pl.grid = (int)((pl.units + pl.per - 1) / pl.per);
+    pl.max_seg = (pl.per + pl.kb - 1) / pl.kb + 1;      // tiles a run of `per` units can touch
+    pl.scratch_elems = (size_t)pl.grid * pl.max_seg * pl.bn * TC_BM;
     return pl;
-}
-
-// Scratch (floats) for the partial sums and counters (ints) a session with `rows` rows needs.
-static inline size_t tc_scratch_elems(size_t rows, int n_sms) {
-    const int bn = 16 << tc_pick_bn((int)std::min<size_t>(rows, 256));
-    return (size_t)2 * n_sms * bn * TC_BM;
-}
-static inline size_t tc_counter_elems(size_t rows, int max_n_out) {
-    return ((size_t)max_n_out / TC_BM + 1) * (rows / 16 + 1);
 }
 
 template <int BN>
@@ -522,20 +398,18 @@ static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& 
                ? RD_OK : RD_E_CUDA;
 }
 
-// Returns RD_E_INVALID_ARG when the shape is not taken (caller falls back to the SIMT kernels).
+// Launches the GEMM; *out describes where a consumer finds the sums.  Returns RD_E_INVALID_ARG when
+// the shape is not taken (caller falls back to the SIMT kernels).
 static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
-                          const TcEpilogue& epi, float* scratch, size_t scratch_elems, int* counters,
-                          size_t counter_elems, int n_sms, int* status, bool chained) {
+                          float* scratch, size_t scratch_elems, int n_sms, int* status, bool chained, PartialSums* out) {
     if (ta.K != K || tw.K != K || tw.n_out != n_out || n_rows < 1 || n_rows > ta.rows) return RD_E_INVALID_ARG;
     const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms);
-    if ((size_t)2 * pl.grid * pl.bn * TC_BM > scratch_elems) return RD_E_INVALID_ARG;
-    if ((size_t)pl.n_tiles_m * pl.n_tiles_n > counter_elems) return RD_E_INVALID_ARG;
+    if (pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
-    p.K = K; p.n_out = n_out; p.n_rows = n_rows;
-    p.kb = pl.kb; p.n_tiles_m = pl.n_tiles_m; p.n_tiles_n = pl.n_tiles_n;
-    p.units = pl.units; p.per = pl.per;
-    p.scratch = scratch; p.counters = counters; p.status = status;
-    p.e = epi;
+    p.kb = pl.kb; p.n_tiles_m = pl.n_tiles_m; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
+    p.scratch = scratch; p.status = status;
+    out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_m = pl.n_tiles_m; out->bn = pl.bn;
+    out->max_seg = pl.max_seg;
     switch (pl.bn_idx) {
         case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);
         case 1: return tc_launch<32>(st, tw.map, ta.map[1], p, pl.grid, chained);

@@ -9,6 +9,7 @@
 #include <stdint.h>
 
 #include "rd_common.cuh"
+#include "rd_partial.cuh"
 
 namespace rd {
 
@@ -162,22 +163,67 @@ __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restr
         x[(size_t)r * hidden + j] = to_f(emb[(size_t)tok * hidden + j]);
 }
 
-// out[row] = g * x / sqrt(mean(x^2) + eps); one block per row.
+// x[row] = src[row] (+ resid[row]);  out[row] = g * x / sqrt(mean(x^2) + eps); one block per row.
+// `src` is a finished array or the partial sums of the GEMM before (added here, in k order);
+// x is kept in shared memory (hidden floats) and, with x_store, written out as the new residual
+// stream (x_store may alias resid).
 template <typename TO>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, size_t ldx, const float* __restrict__ g,
-                               int hidden, float eps, TO* __restrict__ out, size_t ldo,
-                               const int* __restrict__ row_pos) {
-    pdl_enter();
+__global__ void __launch_bounds__(512)
+rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,
+               size_t ldx, const float* __restrict__ g, int hidden, float eps, TO* __restrict__ out, size_t ldo,
+               const int* __restrict__ row_pos) {
+    extern __shared__ __align__(16) float xrow[];
     __shared__ float sm[32];
+    pdl_enter();
     const int r = blockIdx.x;
     if (row_pos && row_pos[r] < 0) return;
-    const float* xr = x + (size_t)r * ldx;
     float ss = 0.f;
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x) ss += xr[j] * xr[j];
+    for (int m = threadIdx.x * 4; m < hidden; m += blockDim.x * 4) {
+        float4 v = row_source_load4(src, r, m);
+        if (resid) {
+            const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
+            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+        if (x_store) *reinterpret_cast<float4*>(x_store + (size_t)r * ldx + m) = v;
+        *reinterpret_cast<float4*>(xrow + m) = v;
+        ss += v.x * v.x;
+        ss += v.y * v.y;
+        ss += v.z * v.z;
+        ss += v.w * v.w;
+    }
     ss = block_sum(ss, sm);
     const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
     for (int j = threadIdx.x; j < hidden; j += blockDim.x)
-        out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xr[j] * inv));
+        out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xrow[j] * inv));
+}
+
+// out[row] = src[row] (+ resid[row]) as a plain float32 array (n multiple of 4: vector path).
+__global__ void reduce_store_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
+                                    float* __restrict__ out, size_t ldo, int n, int n_rows,
+                                    const int* __restrict__ row_pos) {
+    pdl_enter();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((n & 3) == 0) {
+        const size_t quads = (size_t)n / 4;
+        if (i >= (size_t)n_rows * quads) return;
+        const int r = (int)(i / quads), m = (int)(i % quads) * 4;
+        if (row_pos[r] < 0) return;
+        float4 v = row_source_load4(src, r, m);
+        if (resid) {
+            const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
+            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+        *reinterpret_cast<float4*>(out + (size_t)r * ldo + m) = v;
+    } else {
+        const size_t per_row = ((size_t)n + 3) / 4;
+        if (i >= (size_t)n_rows * per_row) return;
+        const int r = (int)(i / per_row), m0 = (int)(i % per_row) * 4;
+        if (row_pos[r] < 0) return;
+        for (int m = m0; m < min(m0 + 4, n); m++) {
+            const float v = row_source_load(src, r, m);
+            out[(size_t)r * ldo + m] = resid ? resid[(size_t)r * ldr + m] + v : v;
+        }
+    }
 }
 
 // act[row] = [ e[row] ; z[row] ] in the GEMM input type (adapter input, Section 3.2).
@@ -236,9 +282,9 @@ gemm_simt_kernel(const T* __restrict__ A, size_t lda, const T* __restrict__ W, i
 
 // Rotary embedding on adjacent pairs of q and k, then: q -> q_t (GEMM/attention input type),
 // k, v -> the row's own cache entry (overwrite: KV-cache sharing, Section 3.2).
-// qkv: [rows, 3h] float32 (q | k | v).  cos/sin: [max_ctx, d/2] float32.
+// src: result of the QKV GEMM, [rows, 3h] (q | k | v).  cos/sin: [max_ctx, d/2] float32.
 template <typename T>
-__global__ void rope_kv_kernel(const float* __restrict__ qkv, const int* __restrict__ row_pos,
+__global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_pos,
                                const int* __restrict__ row_seq, const float* __restrict__ cos_t,
                                const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
                                T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride) {
@@ -247,20 +293,28 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, const int* __restr
     const int p = row_pos[r];
     if (p < 0) return;
     const int half = head_dim / 2;
-    const float* src = qkv + (size_t)r * 3 * hidden;
     T* kdst = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
     T* vdst = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
-    for (int idx = threadIdx.x; idx < hidden / 2; idx += blockDim.x) {
-        const int i = idx % half;
-        const float c = cos_t[(size_t)p * half + i], s = sin_t[(size_t)p * half + i];
-        const float q0 = src[2 * idx], q1 = src[2 * idx + 1];
-        const float k0 = src[hidden + 2 * idx], k1 = src[hidden + 2 * idx + 1];
-        q_t[(size_t)r * hidden + 2 * idx] = from_f<T>(q0 * c - q1 * s);
-        q_t[(size_t)r * hidden + 2 * idx + 1] = from_f<T>(q0 * s + q1 * c);
-        kdst[2 * idx] = from_f<T>(k0 * c - k1 * s);
-        kdst[2 * idx + 1] = from_f<T>(k0 * s + k1 * c);
-        vdst[2 * idx] = from_f<T>(src[2 * hidden + 2 * idx]);
-        vdst[2 * idx + 1] = from_f<T>(src[2 * hidden + 2 * idx + 1]);
+    T* qdst = q_t + (size_t)r * hidden;
+    // four features = two rotary pairs per thread and turn
+    for (int m = (blockIdx.y * blockDim.x + threadIdx.x) * 4; m < hidden; m += gridDim.y * blockDim.x * 4) {
+        const float4 q = row_source_load4(src, r, m), k = row_source_load4(src, r, hidden + m),
+                     v = row_source_load4(src, r, 2 * hidden + m);
+        const int i0 = ((m % head_dim) >> 1), i1 = (((m + 2) % head_dim) >> 1);
+        const float c0 = cos_t[(size_t)p * half + i0], s0 = sin_t[(size_t)p * half + i0];
+        const float c1 = cos_t[(size_t)p * half + i1], s1 = sin_t[(size_t)p * half + i1];
+        qdst[m] = from_f<T>(q.x * c0 - q.y * s0);
+        qdst[m + 1] = from_f<T>(q.x * s0 + q.y * c0);
+        qdst[m + 2] = from_f<T>(q.z * c1 - q.w * s1);
+        qdst[m + 3] = from_f<T>(q.z * s1 + q.w * c1);
+        kdst[m] = from_f<T>(k.x * c0 - k.y * s0);
+        kdst[m + 1] = from_f<T>(k.x * s0 + k.y * c0);
+        kdst[m + 2] = from_f<T>(k.z * c1 - k.w * s1);
+        kdst[m + 3] = from_f<T>(k.z * s1 + k.w * c1);
+        vdst[m] = from_f<T>(v.x);
+        vdst[m + 1] = from_f<T>(v.y);
+        vdst[m + 2] = from_f<T>(v.z);
+        vdst[m + 3] = from_f<T>(v.w);
     }
 }
 
@@ -330,59 +384,71 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
     }
 }
 
-// act[r, j] = silu(gate_j) * up_j.  Plain layout: gu[r] = [gate_0..gate_{I-1} | up_0..up_{I-1}].
-// Interleaved layout (the weight rows were reordered at load for the tensor-core epilogue): groups
-// of 32 = 16 gate features followed by the 16 matching up features.
+// act[r, j..j+3] = silu(gate) * up with gate = acc[r, j], up = acc[r, I + j] of the gate/up GEMM.
 template <typename T>
-__global__ void swiglu_kernel(const float* __restrict__ gu, int inner, T* __restrict__ act, size_t lda,
-                              int n_rows, int interleaved) {
+__global__ void swiglu_kernel(const RowSource src, int inner, T* __restrict__ act, size_t lda, int n_rows,
+                              const int* __restrict__ row_pos) {
     pdl_enter();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= (size_t)n_rows * inner) return;
-    const size_t r = i / inner, j = i % inner;
-    const size_t gi = interleaved ? (j >> 4) * 32 + (j & 15) : j;
-    const size_t ui = interleaved ? gi + 16 : inner + j;
-    const float g = gu[r * 2 * inner + gi], u = gu[r * 2 * inner + ui];
-    act[r * lda + j] = from_f<T>((g / (1.0f + expf(-g))) * u);
+    const size_t quads = (size_t)inner / 4;
+    if (i >= (size_t)n_rows * quads) return;
+    const int r = (int)(i / quads), j = (int)(i % quads) * 4;
+    if (row_pos[r] < 0) return;
+    const float4 g = row_source_load4(src, r, j), u = row_source_load4(src, r, inner + j);
+    const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int k = 0; k < 4; k++) act[(size_t)r * lda + j + k] = from_f<T>((gv[k] / (1.0f + expf(-gv[k]))) * uv[k]);
 }
 
-// Sample(p) of Algorithms 1-2, one block per row.  Greedy: arg max, lowest index on ties.
-// Otherwise Gumbel-max: arg max of logit / T - log(-log u_v), u_v keyed by (seed, sequence,
-// token position, v).  The row at position p drafts the token of position p + 1.
+// Sample(p) of Algorithms 1-2 in two kernels.  Greedy: arg max, lowest index on ties.  Otherwise
+// Gumbel-max: arg max of logit / T - log(-log u_v), u_v keyed by (seed, sequence, token position, v).
+// The row at position p drafts the token of position p + 1.
+//
+// First kernel, grid (rows, chunks): block (r, c) takes the logits of row r (result of the LM-head
+// GEMM, partial sums added here) for the c-th run of `chunk` vocabulary entries (chunk a multiple
+// of 4), optionally stores them, and leaves its best (score, index).
+constexpr int SAMPLE_CHUNKS = 16;
 __global__ void __launch_bounds__(256)
-sample_kernel(const float* __restrict__ logits, int vocab, const int* __restrict__ row_pos,
-              const int* __restrict__ row_seq, float temperature, uint64_t seed, int* __restrict__ draft,
-              int* __restrict__ tokens, int tok_stride) {
-    pdl_enter();
+sample_scan_kernel(const RowSource src, int vocab, int chunk, const int* __restrict__ row_pos,
+                   const int* __restrict__ row_seq, float temperature, uint64_t seed,
+                   float* __restrict__ logits_store, float* __restrict__ best_val, int* __restrict__ best_idx) {
     __shared__ float sv[8];
     __shared__ int si[8];
-    const int r = blockIdx.x;
+    pdl_enter();
+    const int r = blockIdx.x, ck = blockIdx.y;
     const int p = row_pos[r];
     if (p < 0) return;
-    const float* lg = logits + (size_t)r * vocab;
+    const int v0 = ck * chunk, v1 = min(vocab, v0 + chunk);
+    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint32_t seq = (uint32_t)row_seq[r];
     float best = -INFINITY;
     int bi = 0x7fffffff;
-    if (temperature <= 0.f) {
-        for (int v = threadIdx.x; v < vocab; v += blockDim.x) {
-            const float x = lg[v];
-            if (x > best) { best = x; bi = v; }
+    for (int v = v0 + threadIdx.x * 4; v < v1; v += blockDim.x * 4) {
+        float x[4];
+        if (v + 3 < vocab && (vocab & 3) == 0) {
+            const float4 q = row_source_load4(src, r, v);
+            x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+        } else {
+#pragma unroll
+            for (int a = 0; a < 4; a++) x[a] = v + a < vocab ? row_source_load(src, r, v + a) : -INFINITY;
         }
-    } else {
-        const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
-        const int nb = (vocab + 3) / 4;
-        for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
-            const uint4 x = philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)(p + 1), (uint32_t)row_seq[r], STREAM_GUMBEL), key);
-            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+        if (logits_store) {
+#pragma unroll
+            for (int a = 0; a < 4; a++)
+                if (v + a < vocab) logits_store[(size_t)r * vocab + v + a] = x[a];
+        }
+        if (temperature > 0.f) {
+            const uint4 w4 = philox4x32_10(make_uint4((uint32_t)(v >> 2), (uint32_t)(p + 1), seq, STREAM_GUMBEL), key);
+            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int a = 0; a < 4; a++) {
-                const int v = blk * 4 + a;
-                if (v < vocab) {
-                    const float g = -logf(-logf(unit_open(w[a])));
-                    const float sc = __fadd_rn(__fdiv_rn(lg[v], temperature), g);
-                    if (sc > best) { best = sc; bi = v; }
-                }
+                const float g = -logf(-logf(unit_open(w[a])));
+                x[a] = __fadd_rn(__fdiv_rn(x[a], temperature), g);
             }
         }
+#pragma unroll
+        for (int a = 0; a < 4; a++)
+            if (v + a < vocab && x[a] > best) { best = x[a]; bi = v + a; }
     }
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) {
@@ -395,10 +461,30 @@ sample_kernel(const float* __restrict__ logits, int vocab, const int* __restrict
     if (threadIdx.x == 0) {
         for (int w = 1; w < (int)(blockDim.x >> 5); w++)
             if (sv[w] > best || (sv[w] == best && si[w] < bi)) { best = sv[w]; bi = si[w]; }
-        if (bi == 0x7fffffff) bi = 0;                 // all -inf / NaN row: defined result
-        draft[r] = bi;
-        tokens[(size_t)row_seq[r] * tok_stride + p + 1] = bi;
+        best_val[r * SAMPLE_CHUNKS + ck] = best;
+        best_idx[r * SAMPLE_CHUNKS + ck] = bi;
     }
+}
+
+// Second kernel, one thread per row: best of the chunks (lowest index on ties) -> draft.
+__global__ void sample_pick_kernel(const float* __restrict__ best_val, const int* __restrict__ best_idx, int n_chunks,
+                                   int n_rows, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                                   int* __restrict__ draft, int* __restrict__ tokens, int tok_stride) {
+    pdl_enter();
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n_rows) return;
+    const int p = row_pos[r];
+    if (p < 0) return;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int c = 0; c < n_chunks; c++) {
+        const float v = best_val[r * SAMPLE_CHUNKS + c];
+        const int i = best_idx[r * SAMPLE_CHUNKS + c];
+        if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+    }
+    if (bi == 0x7fffffff) bi = 0;                 // all -inf / NaN row: defined result
+    draft[r] = bi;
+    tokens[(size_t)row_seq[r] * tok_stride + p + 1] = bi;
 }
 
 // delta_i = ||z_i - z_prev,i|| / ||z_i||  (Eq. 3); +inf when ||z_i|| = 0.
@@ -474,18 +560,6 @@ template <typename T>
 __global__ void convert_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         dst[i] = from_f<T>(src[i]);
-}
-// Gate/up rows reordered for the fused SwiGLU epilogue: destination row (j/16)*32 + j%16 takes gate
-// feature j, row (j/16)*32 + 16 + j%16 takes up feature j.  src = [gate rows | up rows], K columns.
-template <typename T>
-__global__ void interleave_gate_up_kernel(const T* __restrict__ src, T* __restrict__ dst, int inner, int K) {
-    const size_t n = (size_t)2 * inner * K;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const size_t row = i / K, k = i % K;
-        const size_t j = row % inner;
-        const size_t drow = (j >> 4) * 32 + (j & 15) + (row >= (size_t)inner ? 16 : 0);
-        dst[drow * K + k] = src[i];
-    }
 }
 template <typename T>
 __global__ void widen_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {

@@ -94,7 +94,6 @@ struct rd_model {
     std::vector<LayerW> layers[3];
     TcWeight t_adapter, t_head;
     bool tc_ok = false;
-    bool gu_interleaved = false;   // gate/up rows stored in groups of 16 gate + 16 up (see swiglu_kernel)
     int n_sms = 148;
 };
 
@@ -125,10 +124,9 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
     const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
     float* stage = nullptr;
     size_t stage_n = 0;
-    void* gu_tmp = nullptr;
     int rc = RD_OK;
     int idx = 0;
-    m->gu_interleaved = c.dtype == RD_BF16 && c.mlp_inner % 16 == 0;
+
     auto mat = [&](void* dst, size_t n) -> int { return put_tensor(m, dst, t[idx++], n, elem_bytes, &stage, &stage_n); };
     auto gain = [&](float** dst) -> int {
         RD_TRY(m->mem.get(dst, h * sizeof(float)));
@@ -149,19 +147,8 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
                 if ((rc = mat(L.wo, h * h))) break;
                 if ((rc = gain(&L.g2))) break;
                 if ((rc = m->mem.get(&L.wgu, 2 * I * h * es))) break;
-                if (m->gu_interleaved) {
-                    // [gate | up] into a temporary, then rows regrouped 16 gate + 16 up
-                    if (!gu_tmp && (rc = m->mem.get(&gu_tmp, 2 * I * h * es))) break;
-                    if ((rc = mat(gu_tmp, I * h))) break;
-                    if ((rc = mat((char*)gu_tmp + I * h * es, I * h))) break;
-                    interleave_gate_up_kernel<bf16><<<2048, 256>>>((const bf16*)gu_tmp, (bf16*)L.wgu, (int)I, (int)h);
-                    cudaError_t e = cudaGetLastError();
-                    if (e == cudaSuccess) e = cudaDeviceSynchronize();
-                    if (e != cudaSuccess) { rc = cuda_fail(e, "interleave_gate_up_kernel", __LINE__); break; }
-                } else {
-                    if ((rc = mat(L.wgu, I * h))) break;
-                    if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
-                }
+                if ((rc = mat(L.wgu, I * h))) break;
+                if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
                 if ((rc = m->mem.get(&L.wd, h * I * es))) break;
                 if ((rc = mat(L.wd, h * I))) break;
             }
@@ -179,7 +166,6 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
         }
     } while (0);
     if (stage) cudaFree(stage);
-    if (gu_tmp) m->mem.release(gu_tmp);
     if (rc) return rc;
     // Tensor-core path: TMA descriptors over every weight matrix (bf16 only).
     m->tc_ok = false;
@@ -205,7 +191,7 @@ extern "C" int rd_load(const rd_config* cfg, const void* const* tensors, int32_t
     const rd_config& c = *cfg;
     if (c.hidden <= 0 || c.n_heads <= 0 || c.head_dim <= 0 || c.mlp_inner <= 0 || c.vocab <= 0) return RD_E_INVALID_ARG;
     if (c.hidden != c.n_heads * c.head_dim || c.hidden % 8 || c.mlp_inner % 8) return RD_E_INVALID_ARG;
-    if (c.head_dim % 2 || c.head_dim > 128) return RD_E_INVALID_ARG;
+    if (c.head_dim % 2 || c.head_dim > 128 || c.hidden > 12288) return RD_E_INVALID_ARG;
     if (c.n_prelude < 0 || c.n_core < 1 || c.n_coda < 0) return RD_E_INVALID_ARG;
     if (c.dtype != RD_F32 && c.dtype != RD_BF16) return RD_E_INVALID_ARG;
     if (elem_bytes != 4 && !(elem_bytes == 2 && c.dtype == RD_BF16)) return RD_E_INVALID_ARG;
@@ -246,12 +232,14 @@ struct rd_session {
     int *step_first = nullptr, *step_n = nullptr, *draft = nullptr;
     unsigned long long* counters = nullptr;
     int* status = nullptr;   // device word: non-zero when a bounded wait ran out
-    float *x = nullptr, *qkv = nullptr, *gu = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
+    float *x = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
     float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
     float* tc_scratch = nullptr;   // partial sums of tiles whose K range is shared between CTAs
     size_t tc_scratch_elems = 0;
-    int* tc_counters = nullptr;    // per-tile arrival counters (zero between launches)
-    size_t tc_counter_elems = 0;
+    float* best_val = nullptr;     // per (row, vocabulary chunk): best score and its index
+    int* best_idx = nullptr;
+    float* acc = nullptr;          // output of the plain GEMM kernel, [rows, n_out]
+    size_t acc_elems = 0;
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
     float *att_o = nullptr, *att_ml = nullptr;   // split-KV partials of the windowed attention
     int grp_rows = 0;           // rows per attention query group in the current pass
@@ -332,13 +320,15 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if ((rc = s->mem.get(&s->counters, 8 * sizeof(unsigned long long)))) break;
         if ((rc = s->mem.get(&s->status, 4 * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->x, R * h * sizeof(float)))) break;
-        if ((rc = s->mem.get(&s->qkv, R * 3 * h * sizeof(float)))) break;
-        if ((rc = s->mem.get(&s->gu, R * 2 * I * sizeof(float)))) break;
+        s->acc_elems = std::max(R * std::max<size_t>(std::max<size_t>(3 * h, 2 * I), h), (size_t)s->n_slots * V);
+        if ((rc = s->mem.get(&s->acc, s->acc_elems * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->e, R * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->z, R * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->z_prev, R * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->logits, (size_t)s->n_slots * V * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->delta, R * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->best_val, R * SAMPLE_CHUNKS * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->best_idx, R * SAMPLE_CHUNKS * sizeof(int)))) break;
         // GEMM-input buffers hold at least 256 rows so that the widest TMA row box stays inside
         const size_t Ra = std::max<size_t>(R, 256);
         if ((rc = s->mem.get(&s->act_h, Ra * h * es))) break;
@@ -374,10 +364,18 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
             s->attn_path = 1;
         }
         if (m->tc_ok) {
-            s->tc_scratch_elems = tc_scratch_elems(R, m->n_sms);
+            // scratch for the partial sums: the largest need over the model's GEMM shapes and over
+            // the row counts a pass can have (one row-tile class each)
+            const int shapes[6][2] = {{c.hidden, 3 * c.hidden}, {c.hidden, c.hidden}, {c.hidden, 2 * c.mlp_inner},
+                                      {c.mlp_inner, c.hidden}, {2 * c.hidden, c.hidden}, {c.hidden, c.vocab}};
+            size_t need = 16;
+            for (int nr = 16; ; nr *= 2) {
+                const int rows = std::min<int>(nr, (int)R);
+                for (auto& sh : shapes) need = std::max(need, tc_plan(sh[0], sh[1], rows, m->n_sms).scratch_elems);
+                if (nr >= (int)R) break;
+            }
+            s->tc_scratch_elems = need;
             if ((rc = s->mem.get(&s->tc_scratch, s->tc_scratch_elems * sizeof(float)))) break;
-            s->tc_counter_elems = tc_counter_elems(R, std::max(std::max(3 * c.hidden, 2 * c.mlp_inner), c.vocab));
-            if ((rc = s->mem.get(&s->tc_counters, s->tc_counter_elems * sizeof(int)))) break;
             bool ok = tc_make_act(&s->t_act_h, s->act_h, (int)Ra, c.hidden) == RD_OK;
             ok &= tc_make_act(&s->t_act_2h, s->act_2h, (int)Ra, 2 * c.hidden) == RD_OK;
             ok &= tc_make_act(&s->t_act_i, s->act_i, (int)Ra, c.mlp_inner) == RD_OK;
@@ -421,42 +419,65 @@ extern "C" int rd_set_launch_chaining(rd_session* s, int32_t on) {
         (s)->stats.kernel_launches++;                                                             \
     } while (0)
 
+// x = src (+ resid): a residual stream whose last GEMM term has not been added yet.  The kernel
+// that reads it next adds the term (rd_partial.cuh).
+struct Pending {
+    RowSource src;
+    const float* resid;
+};
+static Pending plain_rows(const float* x, size_t ld) {
+    Pending p = {};
+    p.src.plain = x; p.src.ld = ld; p.resid = nullptr;
+    return p;
+}
+
 template <typename T> struct Eng {
     static bool tc_usable(const rd_session* s, const TcAct* ta, const TcWeight* tw) {
         return sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid;
     }
-    static int tc_run(rd_session* s, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
-                      const TcEpilogue& epi) {
-        const int rc = tc_gemm(s->stream, ta, tw, K, n_out, n_rows, epi, s->tc_scratch, s->tc_scratch_elems,
-                               s->tc_counters, s->tc_counter_elems, s->m->n_sms, s->status, s->chained);
-        if (rc == RD_OK) { s->stats.tc_gemm_launches++; s->stats.kernel_launches++; }
-        else if (rc == RD_E_CUDA) return cuda_fail(cudaGetLastError(), "tensor-core GEMM launch", __LINE__);
-        return rc;
-    }
 
-    // Y[r, o] = sum_k A[r, k] W[o, k] (+ resid[r, o]).  `ta`/`tw` are the operands' TMA descriptors for
-    // the tensor-core path (bf16 only).
+    // acc[r, o] = sum_k A[r, k] W[o, k]; *out tells the consumer where the sums are: partial sums of
+    // the tensor-core kernel, or the finished array s->acc of the plain kernel.
     static int gemm(rd_session* s, const T* A, size_t lda, const TcAct* ta, const T* W, const TcWeight* tw, int K,
-                    int n_out, float* Y, size_t ldy, const float* resid, int n_rows) {
+                    int n_out, int n_rows, RowSource* out) {
         const int br = bracket_open(s, 0, (uint64_t)n_out * K * sizeof(T));
+        *out = RowSource{};
         if (tc_usable(s, ta, tw)) {
-            TcEpilogue e = {};
-            e.mode = TC_EPI_STORE; e.Y = Y; e.ldy = ldy; e.resid = resid; e.ldr = ldy;
-            const int rc = tc_run(s, *ta, *tw, K, n_out, n_rows, e);
-            if (rc == RD_OK) { bracket_close(s, br); return RD_OK; }
+            const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, n_rows, s->tc_scratch, s->tc_scratch_elems, s->m->n_sms,
+                                   s->status, s->chained, &out->part);
+            if (rc == RD_OK) {
+                s->stats.tc_gemm_launches++; s->stats.kernel_launches++;
+                bracket_close(s, br);
+                return RD_OK;
+            }
+            if (rc == RD_E_CUDA) return cuda_fail(cudaGetLastError(), "tensor-core GEMM launch", __LINE__);
             if (rc != RD_E_INVALID_ARG) return rc;   // INVALID_ARG: shape not taken, fall through
         }
+        if ((size_t)n_rows * n_out > s->acc_elems) return RD_E_CAPACITY;
+        float* Y = s->acc;
+        const size_t ldy = n_out;
+        const float* no_resid = nullptr;
         const int warps = 8;
         dim3 grid((n_out + warps - 1) / warps, 1);
         if (n_rows == 1) {
-            LAUNCH(s, (gemm_simt_kernel<T, 1>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 1>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, no_resid, ldy, n_rows);
         } else if (n_rows <= 4) {
-            LAUNCH(s, (gemm_simt_kernel<T, 4>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 4>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, no_resid, ldy, n_rows);
         } else {
             grid.y = (n_rows + 7) / 8;
-            LAUNCH(s, (gemm_simt_kernel<T, 8>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, resid, ldy, n_rows);
+            LAUNCH(s, (gemm_simt_kernel<T, 8>), grid, warps * 32, 0, A, lda, W, K, n_out, Y, ldy, no_resid, ldy, n_rows);
         }
+        out->plain = Y; out->ld = ldy;
         bracket_close(s, br);
+        return RD_OK;
+    }
+
+    // out[row] = RMSNorm(x; g) with x = in.src (+ in.resid); x_store (may be null) receives x.
+    template <typename TO>
+    static int norm(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
+        const int h = s->m->cfg.hidden;
+        LAUNCH(s, rmsnorm_kernel<TO>, n_rows, 512, (size_t)h * sizeof(float), in.src, in.resid, (size_t)h, x_store, (size_t)h,
+               g, h, s->m->cfg.norm_eps, out, (size_t)h, s->row_pos);
         return RD_OK;
     }
 
@@ -490,35 +511,23 @@ template <typename T> struct Eng {
         }
     }
 
-    // One transformer layer over the rows of the current row table: reads x_in, leaves the
-    // mid-layer residual in s->x, writes x_out (x_in, x_out may both be s->x).
-    static int layer(rd_session* s, int blk, int l, const float* x_in, float* x_out, int n_rows) {
+    // One transformer layer over the rows of the current row table.  Input x = in.src (+ in.resid);
+    // the result is returned pending: x_out = s->x + (down-projection sums), added by whoever reads it.
+    static int layer(rd_session* s, int blk, int l, const Pending& in, Pending* out, int n_rows) {
         const rd_config& c = s->m->cfg;
         const LayerW& L = s->m->layers[blk][l];
         const int h = c.hidden, I = c.mlp_inner;
         const size_t layer_off = (size_t)l * s->sc.batch * s->seq_stride;
         T* Kc = (T*)s->Kc[blk] + layer_off;
         T* Vc = (T*)s->Vc[blk] + layer_off;
-        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, x_in, (size_t)h, L.g1, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
-        // q, k, v: on the tensor-core path the rotary embedding and the cache write are the GEMM's epilogue
-        bool qkv_done = false;
-        if constexpr (sizeof(T) == 2) {
-            if (tc_usable(s, &s->t_act_h, &L.t_qkv)) {
-                const int br = bracket_open(s, 0, (uint64_t)3 * h * h * sizeof(T));
-                TcEpilogue e = {};
-                e.mode = TC_EPI_QKV; e.q_t = (bf16*)s->q_t; e.Kc = (bf16*)Kc; e.Vc = (bf16*)Vc; e.seq_stride = s->seq_stride;
-                e.hidden = h; e.head_dim = c.head_dim; e.row_pos = s->row_pos; e.row_seq = s->row_seq;
-                e.cos_t = s->cos_t; e.sin_t = s->sin_t;
-                const int rc = tc_run(s, s->t_act_h, L.t_qkv, h, 3 * h, n_rows, e);
-                if (rc == RD_OK) { bracket_close(s, br); qkv_done = true; }
-                else if (rc != RD_E_INVALID_ARG) return rc;
-            }
-        }
-        if (!qkv_done) {
-            RD_TRY(gemm(s, (T*)s->act_h, h, nullptr, (T*)L.wqkv, nullptr, h, 3 * h, s->qkv, 3 * h, nullptr, n_rows));
-            LAUNCH(s, rope_kv_kernel<T>, n_rows, 256, 0, s->qkv, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
-                   (T*)s->q_t, Kc, Vc, s->seq_stride);
-        }
+        // x_in is materialised in s->x unless it already is a finished array
+        const bool lazy = in.resid != nullptr || in.src.plain == nullptr;
+        RD_TRY(norm<T>(s, in, lazy ? s->x : nullptr, L.g1, (T*)s->act_h, n_rows));
+        const float* x_in = lazy ? s->x : in.src.plain;
+        RowSource acc;
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
+        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 4), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+               (T*)s->q_t, Kc, Vc, s->seq_stride);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
         if constexpr (sizeof(T) == 2) {
@@ -532,27 +541,22 @@ template <typename T> struct Eng {
                    s->seq_stride, h, c.head_dim, (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
         }
         bracket_close(s, br);
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, s->x, h, x_in, n_rows));
-        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, s->x, (size_t)h, L.g2, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
-        // gate/up: with interleaved weight rows SwiGLU is the GEMM's epilogue
-        bool mlp_done = false;
-        if constexpr (sizeof(T) == 2) {
-            if (s->m->gu_interleaved && tc_usable(s, &s->t_act_h, &L.t_gu)) {
-                const int br2 = bracket_open(s, 0, (uint64_t)2 * I * h * sizeof(T));
-                TcEpilogue e = {};
-                e.mode = TC_EPI_SWIGLU; e.act = (bf16*)s->act_i; e.lda = I; e.inner = I;
-                const int rc = tc_run(s, s->t_act_h, L.t_gu, h, 2 * I, n_rows, e);
-                if (rc == RD_OK) { bracket_close(s, br2); mlp_done = true; }
-                else if (rc != RD_E_INVALID_ARG) return rc;
-            }
-        }
-        if (!mlp_done) {
-            RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, s->gu, 2 * I, nullptr, n_rows));
-            const size_t n_el = (size_t)n_rows * I;
-            LAUNCH(s, swiglu_kernel<T>, (unsigned)((n_el + 255) / 256), 256, 0, s->gu, I, (T*)s->act_i, (size_t)I, n_rows,
-                   s->m->gu_interleaved ? 1 : 0);
-        }
-        RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, x_out, h, s->x, n_rows));
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, n_rows, &acc));
+        Pending mid = {acc, x_in};                      // x_mid = x_in + out-projection, stored in s->x
+        RD_TRY(norm<T>(s, mid, s->x, L.g2, (T*)s->act_h, n_rows));
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, n_rows, &acc));
+        const size_t n_q = (size_t)n_rows * (I / 4);
+        LAUNCH(s, swiglu_kernel<T>, (unsigned)((n_q + 255) / 256), 256, 0, acc, I, (T*)s->act_i, (size_t)I, n_rows, s->row_pos);
+        RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, n_rows, &out->src));
+        out->resid = s->x;
+        return RD_OK;
+    }
+
+    // dst[row] = x[row] for a pending x.
+    static int materialise(rd_session* s, const Pending& in, float* dst, int n, int n_rows) {
+        const size_t items = (size_t)n_rows * ((n + 3) / 4);
+        LAUNCH(s, reduce_store_kernel, (unsigned)((items + 255) / 256), 256, 0, in.src, in.resid, (size_t)n, dst, (size_t)n, n,
+               n_rows, s->row_pos);
         return RD_OK;
     }
 
@@ -562,8 +566,14 @@ template <typename T> struct Eng {
         float* x0 = c.n_prelude > 0 ? s->x : e_out;
         LAUNCH(s, embed_kernel<T>, n_rows, 256, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride, (const T*)s->m->emb,
                c.hidden, x0);
-        for (int l = 0; l < c.n_prelude; l++) RD_TRY(layer(s, 0, l, s->x, l == c.n_prelude - 1 ? e_out : s->x, n_rows));
-        return RD_OK;
+        if (c.n_prelude == 0) return RD_OK;
+        Pending x = plain_rows(s->x, c.hidden);
+        for (int l = 0; l < c.n_prelude; l++) {
+            Pending y;
+            RD_TRY(layer(s, 0, l, x, &y, n_rows));
+            x = y;
+        }
+        return materialise(s, x, e_out, c.hidden, n_rows);
     }
 
     // z_out = R(e, z_in): adapter over concat(e, z), core layers, closing RMSNorm.
@@ -571,25 +581,42 @@ template <typename T> struct Eng {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
         LAUNCH(s, concat_kernel<T>, n_rows, 256, 0, e, (size_t)h, z_in, (size_t)h, h, (T*)s->act_2h, (size_t)2 * h, s->row_pos);
-        RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, s->x, h,
-                    nullptr, n_rows));
-        for (int l = 0; l < c.n_core; l++) RD_TRY(layer(s, 1, l, s->x, s->x, n_rows));
-        LAUNCH(s, rmsnorm_kernel<float>, n_rows, 256, 0, s->x, (size_t)h, s->m->g_core, h, c.norm_eps, z_out, (size_t)h, s->row_pos);
-        return RD_OK;
+        Pending x = {};
+        RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, n_rows, &x.src));
+        if (x.src.plain) {
+            // finished sums sit in the plain kernel's output buffer, which the next GEMM overwrites
+            RD_TRY(materialise(s, x, s->x, h, n_rows));
+            x = plain_rows(s->x, h);
+        }
+        for (int l = 0; l < c.n_core; l++) {
+            Pending y;
+            RD_TRY(layer(s, 1, l, x, &y, n_rows));
+            x = y;
+        }
+        return norm<float>(s, x, nullptr, s->m->g_core, z_out, n_rows);
     }
 
     // Coda layers on x = z; with `head`: final RMSNorm, LM head, Sample -> drafts.
     static int coda(rd_session* s, const float* z, int n_rows, bool head) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
-        for (int l = 0; l < c.n_coda; l++) RD_TRY(layer(s, 2, l, l == 0 ? z : s->x, s->x, n_rows));
-        if (!head) return RD_OK;
-        const float* xf = c.n_coda > 0 ? s->x : z;
-        LAUNCH(s, rmsnorm_kernel<T>, n_rows, 256, 0, xf, (size_t)h, s->m->g_final, h, c.norm_eps, (T*)s->act_h, (size_t)h, s->row_pos);
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, s->logits, c.vocab,
-                    nullptr, n_rows));
-        LAUNCH(s, sample_kernel, n_rows, 256, 0, s->logits, c.vocab, s->row_pos, s->row_seq, s->sc.temperature, s->sc.seed,
-               s->draft, s->tokens, s->tok_stride);
+        Pending x = plain_rows(z, h);
+        for (int l = 0; l < c.n_coda; l++) {
+            Pending y;
+            RD_TRY(layer(s, 2, l, x, &y, n_rows));
+            x = y;
+        }
+        if (!head) return RD_OK;     // (the last layer's pending sums are not needed: only its K/V were)
+        RD_TRY(norm<T>(s, x, nullptr, s->m->g_final, (T*)s->act_h, n_rows));
+        RowSource lg;
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, n_rows, &lg));
+        // vocabulary split into at most SAMPLE_CHUNKS runs (multiples of 4) per row
+        const int chunk = ((c.vocab + SAMPLE_CHUNKS - 1) / SAMPLE_CHUNKS + 3) / 4 * 4;
+        const int n_chunks = (c.vocab + chunk - 1) / chunk;
+        LAUNCH(s, sample_scan_kernel, dim3(n_rows, n_chunks), 256, 0, lg, c.vocab, chunk, s->row_pos, s->row_seq,
+               s->sc.temperature, s->sc.seed, s->sc.keep_logits ? s->logits : (float*)nullptr, s->best_val, s->best_idx);
+        LAUNCH(s, sample_pick_kernel, (n_rows + 63) / 64, 64, 0, s->best_val, s->best_idx, n_chunks, n_rows, s->row_pos,
+               s->row_seq, s->draft, s->tokens, s->tok_stride);
         return RD_OK;
     }
 

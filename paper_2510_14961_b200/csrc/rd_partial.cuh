@@ -1,0 +1,59 @@
+// Where the consumer of a GEMM finds the GEMM's result.
+//
+// The tensor-core GEMM (rd_gemm_tc.cuh) cuts the k range of a 128-feature tile between CTAs and
+// leaves one slot of fp32 partial sums per (CTA, tile it touched).  The kernel that consumes the
+// result adds the slots of a tile in ascending k order while it reads: the order is fixed by the
+// shapes alone, so results are bit-reproducible.  The plain GEMM kernel writes finished sums to an
+// ordinary [rows, n_out] array instead; RowSource covers both.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace rd {
+
+// Units (tile, k-block) are numbered tile by tile, kb per tile; CTA g owns units [g*per, (g+1)*per).
+// The j-th tile CTA g touches went to slot g*max_seg + j, laid out [bn rows][128 features].
+struct PartialSums {
+    const float* scratch;
+    int kb, per, n_tiles_m, bn, max_seg;
+};
+
+struct RowSource {
+    const float* plain;   // non-null: value(r, m) = plain[r * ld + m]
+    size_t ld;
+    PartialSums part;     // otherwise: sum of the tile's slots
+};
+
+// Sum of features m..m+3 (m a multiple of 4) of row r.
+__device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, int m) {
+    if (s.plain) return *reinterpret_cast<const float4*>(s.plain + (size_t)r * s.ld + m);
+    const PartialSums& d = s.part;
+    const int tile = (r / d.bn) * d.n_tiles_m + (m >> 7);
+    const long long t_lo = (long long)tile * d.kb;
+    const int g_lo = (int)(t_lo / d.per), g_hi = (int)((t_lo + d.kb - 1) / d.per);
+    const size_t in_slot = (size_t)(r % d.bn) * 128 + (m & 127);
+    const float* base = d.scratch + in_slot;
+    const size_t slot_elems = (size_t)d.bn * 128;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // slots are requested four at a time (one round trip to L2), then added in ascending k order
+    for (int gb = g_lo; gb <= g_hi; gb += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            const int g = min(gb + q, g_hi);
+            const int first_tile = (int)(((long long)g * d.per) / d.kb);
+            v[q] = __ldcg(reinterpret_cast<const float4*>(base + ((size_t)g * d.max_seg + (tile - first_tile)) * slot_elems));
+        }
+#pragma unroll
+        for (int q = 0; q < 4; q++)
+            if (gb + q <= g_hi) { acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w; }
+    }
+    return acc;
+}
+__device__ __forceinline__ float row_source_load(const RowSource& s, int r, int m) {
+    if (s.plain) return s.plain[(size_t)r * s.ld + m];
+    const float4 v = row_source_load4(s, r, m & ~3);
+    const int k = m & 3;
+    return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
+}
+
+}  // namespace rd
