@@ -6,6 +6,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <cooperative_groups.h>
 #include <stdint.h>
 
 #include "rd_common.cuh"
@@ -149,52 +150,69 @@ __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __
     }
 }
 
-// x[row] = emb[token at the row's position]
+// x[row] = emb[token at the row's position]; grid (rows, parts), 16-byte loads.
 template <typename T>
 __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                              const int* __restrict__ tokens, int tok_stride, const T* __restrict__ emb,
                              int hidden, float* __restrict__ x) {
     pdl_enter();
+    constexpr int VEC = Vec16<T>::N;
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
     const int tok = tokens[(size_t)row_seq[r] * tok_stride + p];
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x)
-        x[(size_t)r * hidden + j] = to_f(emb[(size_t)tok * hidden + j]);
+    for (int j = (blockIdx.y * blockDim.x + threadIdx.x) * VEC; j < hidden; j += gridDim.y * blockDim.x * VEC) {
+        float v[VEC];
+        Vec16<T>::load(emb + (size_t)tok * hidden + j, v);
+#pragma unroll
+        for (int i = 0; i < VEC; i++) x[(size_t)r * hidden + j + i] = v[i];
+    }
 }
 
-// x[row] = src[row] (+ resid[row]);  out[row] = g * x / sqrt(mean(x^2) + eps); one block per row.
-// `src` is a finished array or the partial sums of the GEMM before (added here, in k order);
-// x is kept in shared memory (hidden floats) and, with x_store, written out as the new residual
-// stream (x_store may alias resid).
+// x[row] = src[row] (+ resid[row]);  out[row] = g * x / sqrt(mean(x^2) + eps).
+// One cluster of NORM_CLUSTER blocks per row, grid (NORM_CLUSTER, rows): each block takes a run of
+// features, keeps its part of x in shared memory, and the blocks exchange their sums of squares
+// through distributed shared memory (added in block order).  `src` is a finished array or the
+// partial sums of the GEMM before (added here, in k order); with x_store, x is written out as the
+// new residual stream (x_store may alias resid).
+constexpr int NORM_CLUSTER = 8;
 template <typename TO>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(256)
 rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,
                size_t ldx, const float* __restrict__ g, int hidden, float eps, TO* __restrict__ out, size_t ldo,
                const int* __restrict__ row_pos) {
-    extern __shared__ __align__(16) float xrow[];
+    extern __shared__ __align__(16) float xpart[];
     __shared__ float sm[32];
+    __shared__ float ss_own;
     pdl_enter();
-    const int r = blockIdx.x;
-    if (row_pos && row_pos[r] < 0) return;
+    cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+    const int r = blockIdx.y;
+    if (row_pos && row_pos[r] < 0) return;                       // the whole cluster leaves
+    const int chunk = ((hidden / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
+    const int m0 = blockIdx.x * chunk, m1 = min(hidden, m0 + chunk);
     float ss = 0.f;
-    for (int m = threadIdx.x * 4; m < hidden; m += blockDim.x * 4) {
+    for (int m = m0 + threadIdx.x * 4; m < m1; m += blockDim.x * 4) {
         float4 v = row_source_load4(src, r, m);
         if (resid) {
             const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
         }
         if (x_store) *reinterpret_cast<float4*>(x_store + (size_t)r * ldx + m) = v;
-        *reinterpret_cast<float4*>(xrow + m) = v;
+        *reinterpret_cast<float4*>(xpart + (m - m0)) = v;
         ss += v.x * v.x;
         ss += v.y * v.y;
         ss += v.z * v.z;
         ss += v.w * v.w;
     }
     ss = block_sum(ss, sm);
-    const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x)
-        out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xrow[j] * inv));
+    if (threadIdx.x == 0) ss_own = ss;
+    cluster.sync();
+    float tot = 0.f;
+    for (int k = 0; k < NORM_CLUSTER; k++) tot += *cluster.map_shared_rank(&ss_own, k);
+    cluster.sync();                                              // no block leaves while its sum may be read
+    const float inv = 1.0f / sqrtf(tot / (float)hidden + eps);
+    for (int j = m0 + threadIdx.x; j < m1; j += blockDim.x)
+        out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xpart[j - m0] * inv));
 }
 
 // out[row] = src[row] (+ resid[row]) as a plain float32 array (n multiple of 4: vector path).
@@ -234,9 +252,13 @@ __global__ void concat_kernel(const float* __restrict__ e, size_t lde, const flo
     pdl_enter();
     const int r = blockIdx.x;
     if (row_pos[r] < 0) return;
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
-        act[(size_t)r * lda + j] = from_f<T>(e[(size_t)r * lde + j]);
-        act[(size_t)r * lda + hidden + j] = from_f<T>(z[(size_t)r * ldz + j]);
+    for (int j = (blockIdx.y * blockDim.x + threadIdx.x) * 4; j < hidden; j += gridDim.y * blockDim.x * 4) {
+        const float4 a = *reinterpret_cast<const float4*>(e + (size_t)r * lde + j);
+        const float4 b = *reinterpret_cast<const float4*>(z + (size_t)r * ldz + j);
+        T* d0 = act + (size_t)r * lda + j;
+        T* d1 = d0 + hidden;
+        d0[0] = from_f<T>(a.x); d0[1] = from_f<T>(a.y); d0[2] = from_f<T>(a.z); d0[3] = from_f<T>(a.w);
+        d1[0] = from_f<T>(b.x); d1[1] = from_f<T>(b.y); d1[2] = from_f<T>(b.z); d1[3] = from_f<T>(b.w);
     }
 }
 

@@ -412,6 +412,12 @@ extern "C" int rd_set_launch_chaining(rd_session* s, int32_t on) {
 // The schedule (templated on the storage type T of weights / KV / GEMM inputs)
 // ---------------------------------------------------------------------------------------------
 // Every kernel of a step is a link of one programmatic-dependent-launch chain (rd_common.cuh).
+#define LAUNCH_CLUSTER(s, kern, grid, block, smem, cluster_x, ...)                                 \
+    do {                                                                                          \
+        cudaError_t e_ = launch_chained_cluster(kern, dim3 grid, dim3(block), smem, (s)->stream, (s)->chained, cluster_x, __VA_ARGS__); \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #kern, __LINE__);                             \
+        (s)->stats.kernel_launches++;                                                             \
+    } while (0)
 #define LAUNCH(s, kern, grid, block, smem, ...)                                                   \
     do {                                                                                          \
         cudaError_t e_ = launch_chained(kern, dim3(grid), dim3(block), smem, (s)->stream, (s)->chained, __VA_ARGS__); \
@@ -476,8 +482,9 @@ template <typename T> struct Eng {
     template <typename TO>
     static int norm(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
         const int h = s->m->cfg.hidden;
-        LAUNCH(s, rmsnorm_kernel<TO>, n_rows, 512, (size_t)h * sizeof(float), in.src, in.resid, (size_t)h, x_store, (size_t)h,
-               g, h, s->m->cfg.norm_eps, out, (size_t)h, s->row_pos);
+        const size_t part = (size_t)((h / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
+        LAUNCH_CLUSTER(s, rmsnorm_kernel<TO>, (NORM_CLUSTER, n_rows), 256, part * sizeof(float), NORM_CLUSTER, in.src, in.resid,
+                       (size_t)h, x_store, (size_t)h, g, h, s->m->cfg.norm_eps, out, (size_t)h, s->row_pos);
         return RD_OK;
     }
 
@@ -526,7 +533,7 @@ template <typename T> struct Eng {
         const float* x_in = lazy ? s->x : in.src.plain;
         RowSource acc;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
-        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 4), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
                (T*)s->q_t, Kc, Vc, s->seq_stride);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
@@ -564,7 +571,7 @@ template <typename T> struct Eng {
     static int prelude(rd_session* s, int n_rows, float* e_out) {
         const rd_config& c = s->m->cfg;
         float* x0 = c.n_prelude > 0 ? s->x : e_out;
-        LAUNCH(s, embed_kernel<T>, n_rows, 256, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride, (const T*)s->m->emb,
+        LAUNCH(s, embed_kernel<T>, dim3(n_rows, 4), 128, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride, (const T*)s->m->emb,
                c.hidden, x0);
         if (c.n_prelude == 0) return RD_OK;
         Pending x = plain_rows(s->x, c.hidden);
@@ -580,7 +587,7 @@ template <typename T> struct Eng {
     static int core(rd_session* s, const float* e, const float* z_in, float* z_out, int n_rows) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
-        LAUNCH(s, concat_kernel<T>, n_rows, 256, 0, e, (size_t)h, z_in, (size_t)h, h, (T*)s->act_2h, (size_t)2 * h, s->row_pos);
+        LAUNCH(s, concat_kernel<T>, dim3(n_rows, 8), 128, 0, e, (size_t)h, z_in, (size_t)h, h, (T*)s->act_2h, (size_t)2 * h, s->row_pos);
         Pending x = {};
         RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, n_rows, &x.src));
         if (x.src.plain) {

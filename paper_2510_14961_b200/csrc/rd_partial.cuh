@@ -27,9 +27,10 @@ struct RowSource {
 __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, int m) {
     if (s.plain) return *reinterpret_cast<const float4*>(s.plain + (size_t)r * s.ld + m);
     const PartialSums& d = s.part;
-    const int tile = (r / d.bn) * d.n_tiles_m + (m >> 7);
-    const long long t_lo = (long long)tile * d.kb;
-    const int g_lo = (int)(t_lo / d.per), g_hi = (int)((t_lo + d.kb - 1) / d.per);
+    // (unit numbers stay far below 2^31: 32-bit arithmetic)
+    const unsigned tile = (unsigned)(r / d.bn) * d.n_tiles_m + (m >> 7);
+    const unsigned t_lo = tile * (unsigned)d.kb;
+    const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
     const size_t in_slot = (size_t)(r % d.bn) * 128 + (m & 127);
     const float* base = d.scratch + in_slot;
     const size_t slot_elems = (size_t)d.bn * 128;
@@ -40,7 +41,7 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
 #pragma unroll
         for (int q = 0; q < 4; q++) {
             const int g = min(gb + q, g_hi);
-            const int first_tile = (int)(((long long)g * d.per) / d.kb);
+            const unsigned first_tile = ((unsigned)g * (unsigned)d.per) / (unsigned)d.kb;
             v[q] = __ldcg(reinterpret_cast<const float4*>(base + ((size_t)g * d.max_seg + (tile - first_tile)) * slot_elems));
         }
 #pragma unroll
