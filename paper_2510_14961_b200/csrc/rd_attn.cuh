@@ -218,27 +218,49 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
 }
 
 // out[row, head*D + e] = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), splits in ascending order.
+// Block = (row, group of 4 heads), one thread per 4 output elements; the (max, sum) pairs and the
+// partial outputs of all splits are requested before any is used.
 template <int D>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_splits,
-                                    const int* __restrict__ row_pos, int hidden, __nv_bfloat16* __restrict__ out) {
+                                    const int* __restrict__ row_pos, int hidden, int n_heads,
+                                    __nv_bfloat16* __restrict__ out) {
     pdl_enter();
-    const int r = blockIdx.x, hd = blockIdx.y, H = gridDim.y;
-    const int e = threadIdx.x;
-    if (e >= D) return;
+    constexpr int Q = D / 4;
+    const int r = blockIdx.x;
+    const int hd = blockIdx.y * 4 + threadIdx.x / Q, e = (threadIdx.x % Q) * 4;
+    if (hd >= n_heads) return;
     __nv_bfloat16* dst = out + (size_t)r * hidden + hd * D + e;
-    if (row_pos[r] < 0) { *dst = __float2bfloat16_rn(0.f); return; }
-    const size_t base = ((size_t)r * H + hd) * n_splits;
-    float M = -INFINITY;
-    for (int s = 0; s < n_splits; s++) M = fmaxf(M, part_ml[(base + s) * 2]);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < n_splits; s++) {
-        const float m = part_ml[(base + s) * 2];
-        if (m == -INFINITY) continue;
-        const float w = exp2f(m - M);
-        num += part_o[(base + s) * D + e] * w;
-        den += part_ml[(base + s) * 2 + 1] * w;
+    if (row_pos[r] < 0) {
+        dst[0] = dst[1] = dst[2] = dst[3] = __float2bfloat16_rn(0.f);
+        return;
     }
-    *dst = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+    const size_t base = ((size_t)r * n_heads + hd) * n_splits;
+    float2 ml[ATT_MAX_SPLITS];
+    float4 o[ATT_MAX_SPLITS];
+#pragma unroll
+    for (int s = 0; s < ATT_MAX_SPLITS; s++) {
+        const int ss = min(s, n_splits - 1);
+        ml[s] = __ldcg(reinterpret_cast<const float2*>(part_ml + (base + ss) * 2));
+        o[s] = __ldcg(reinterpret_cast<const float4*>(part_o + (base + ss) * D + e));
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < ATT_MAX_SPLITS; s++)
+        if (s < n_splits) M = fmaxf(M, ml[s].x);
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+#pragma unroll
+    for (int s = 0; s < ATT_MAX_SPLITS; s++) {
+        if (s >= n_splits || ml[s].x == -INFINITY) continue;
+        const float w = exp2f(ml[s].x - M);
+        num.x += o[s].x * w; num.y += o[s].y * w; num.z += o[s].z * w; num.w += o[s].w * w;
+        den += ml[s].y * w;
+    }
+    const float inv = den > 0.f ? 1.0f / den : 0.f;
+    dst[0] = __float2bfloat16_rn(num.x * inv);
+    dst[1] = __float2bfloat16_rn(num.y * inv);
+    dst[2] = __float2bfloat16_rn(num.z * inv);
+    dst[3] = __float2bfloat16_rn(num.w * inv);
 }
 
 }  // namespace rd

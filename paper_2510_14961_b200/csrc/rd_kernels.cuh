@@ -183,11 +183,14 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
                const int* __restrict__ row_pos) {
     extern __shared__ __align__(16) float xpart[];
     __shared__ float sm[32];
-    __shared__ float ss_own;
+    __shared__ float ss_all[NORM_CLUSTER];                       // every block's sum, pushed by its owner
     pdl_enter();
     cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
     const int r = blockIdx.y;
     if (row_pos && row_pos[r] < 0) return;                       // the whole cluster leaves
+    // first cluster barrier, split: arrive now, wait before the first access to another block's
+    // shared memory (which is only legal once that block runs)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     const int chunk = ((hidden / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
     const int m0 = blockIdx.x * chunk, m1 = min(hidden, m0 + chunk);
     float ss = 0.f;
@@ -205,11 +208,13 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
         ss += v.w * v.w;
     }
     ss = block_sum(ss, sm);
-    if (threadIdx.x == 0) ss_own = ss;
+    // each block writes its sum into every block's table; after the cluster barrier all tables are
+    // complete and nobody touches another block's memory again
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (threadIdx.x < NORM_CLUSTER) *cluster.map_shared_rank(&ss_all[blockIdx.x], threadIdx.x) = ss;
     cluster.sync();
     float tot = 0.f;
-    for (int k = 0; k < NORM_CLUSTER; k++) tot += *cluster.map_shared_rank(&ss_own, k);
-    cluster.sync();                                              // no block leaves while its sum may be read
+    for (int k = 0; k < NORM_CLUSTER; k++) tot += ss_all[k];
     const float inv = 1.0f / sqrtf(tot / (float)hidden + eps);
     for (int j = m0 + threadIdx.x; j < m1; j += blockDim.x)
         out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xpart[j - m0] * inv));

@@ -282,6 +282,47 @@ static void bracket_close(rd_session* s, int idx) {
     if (idx >= 0) cudaEventRecord(s->brackets[idx].b, s->stream);
 }
 
+// The GEMM kernels need the largest shared-memory carve-out an SM offers.  Every other kernel of a
+// step asks for the same carve-out, so that an SM never has to drain and switch its L1 / shared
+// split between two kernels of the chain, and a kernel launched early can share an SM with its
+// predecessor.
+template <typename F> static void want_max_carveout(F* kern) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+template <typename T> static void want_max_carveout_typed() {
+    want_max_carveout(embed_kernel<T>);
+    want_max_carveout(rmsnorm_kernel<T>);
+    want_max_carveout(concat_kernel<T>);
+    want_max_carveout(gemm_simt_kernel<T, 1>);
+    want_max_carveout(gemm_simt_kernel<T, 4>);
+    want_max_carveout(gemm_simt_kernel<T, 8>);
+    want_max_carveout(rope_kv_kernel<T>);
+    want_max_carveout(attn_row_kernel<T>);
+    want_max_carveout(swiglu_kernel<T>);
+}
+static void want_max_carveout_everywhere() {
+    static bool done = false;
+    if (done) return;
+    done = true;
+    want_max_carveout_typed<float>();
+    want_max_carveout_typed<bf16>();
+    want_max_carveout(plan_rows_kernel);
+    want_max_carveout(fill_rows_kernel);
+    want_max_carveout(init_state_kernel);
+    want_max_carveout(reduce_store_kernel);
+    want_max_carveout(sample_scan_kernel);
+    want_max_carveout(sample_pick_kernel);
+    want_max_carveout(delta_kernel);
+    want_max_carveout(advance_kernel);
+    want_max_carveout(attn_window_kernel<64>);
+    want_max_carveout(attn_window_kernel<96>);
+    want_max_carveout(attn_window_kernel<128>);
+    want_max_carveout(attn_combine_kernel<64>);
+    want_max_carveout(attn_combine_kernel<96>);
+    want_max_carveout(attn_combine_kernel<128>);
+    cudaGetLastError();   // an attribute a kernel does not take is not an error of the session
+}
+
 extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp, void* cuda_stream,
                                  rd_session** out) {
     if (!m || !scp || !out) return RD_E_INVALID_ARG;
@@ -291,6 +332,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
     rd_session* s = new (std::nothrow) rd_session();
     if (!s) return RD_E_OOM;
+    want_max_carveout_everywhere();
     s->m = m;
     s->sc = sc;
     s->stream = (cudaStream_t)cuda_stream;
@@ -359,8 +401,8 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if (e == cudaSuccess) e = cudaMemcpy(s->done, ones.data(), B * sizeof(int), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { rc = cuda_fail(e, "session init copies", __LINE__); break; }
         if (c.dtype == RD_BF16 && (c.head_dim == 64 || c.head_dim == 96 || c.head_dim == 128)) {
-            if ((rc = s->mem.get(&s->att_o, R * c.n_heads * 8 * (size_t)c.head_dim * sizeof(float)))) break;
-            if ((rc = s->mem.get(&s->att_ml, R * c.n_heads * 8 * 2 * sizeof(float)))) break;
+            if ((rc = s->mem.get(&s->att_o, R * c.n_heads * ATT_MAX_SPLITS * (size_t)c.head_dim * sizeof(float)))) break;
+            if ((rc = s->mem.get(&s->att_ml, R * c.n_heads * ATT_MAX_SPLITS * 2 * sizeof(float)))) break;
             s->attn_path = 1;
         }
         if (m->tc_ok) {
@@ -499,14 +541,15 @@ template <typename T> struct Eng {
         const rd_config& c = s->m->cfg;
         const int groups = (n_rows + s->grp_rows - 1) / s->grp_rows;
         const int tiles = std::max(1, (s->ctx_max + ATT_KT - 1) / ATT_KT);
+        // enough (group, head, split) blocks for two per SM; a split never gets less than one tile
         int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
         ns = std::max(1, std::min(std::min(ns, 8), tiles));
         const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
         LAUNCH(s, attn_window_kernel<D>, dim3(c.n_heads, groups, ns), 128, AttCfg<D>::SMEM, (const bf16*)s->q_t,
                s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden, scale_log2, ns, s->att_o,
                s->att_ml);
-        LAUNCH(s, attn_combine_kernel<D>, dim3(n_rows, c.n_heads), D, 0, s->att_o, s->att_ml, ns, s->row_pos, c.hidden,
-               (bf16*)s->act_h);
+        LAUNCH(s, attn_combine_kernel<D>, dim3(n_rows, (c.n_heads + 3) / 4), D, 0, s->att_o, s->att_ml, ns, s->row_pos,
+               c.hidden, c.n_heads, (bf16*)s->act_h);
         return RD_OK;
     }
     static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {

@@ -35,17 +35,20 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     const float* base = d.scratch + in_slot;
     const size_t slot_elems = (size_t)d.bn * 128;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    // slots are requested four at a time (one round trip to L2), then added in ascending k order
-    for (int gb = g_lo; gb <= g_hi; gb += 4) {
-        float4 v[4];
+    // up to eight slots are requested together (one round trip to L2), then added in ascending k order
+    for (int gb = g_lo; gb <= g_hi; gb += 8) {
+        float4 v[8];
 #pragma unroll
-        for (int q = 0; q < 4; q++) {
-            const int g = min(gb + q, g_hi);
-            const unsigned first_tile = ((unsigned)g * (unsigned)d.per) / (unsigned)d.kb;
-            v[q] = __ldcg(reinterpret_cast<const float4*>(base + ((size_t)g * d.max_seg + (tile - first_tile)) * slot_elems));
+        for (int q = 0; q < 8; q++) {
+            v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (gb + q <= g_hi) {
+                const unsigned g = (unsigned)(gb + q);
+                const unsigned first_tile = (g * (unsigned)d.per) / (unsigned)d.kb;
+                v[q] = __ldcg(reinterpret_cast<const float4*>(base + ((size_t)g * d.max_seg + (tile - first_tile)) * slot_elems));
+            }
         }
 #pragma unroll
-        for (int q = 0; q < 4; q++)
+        for (int q = 0; q < 8; q++)
             if (gb + q <= g_hi) { acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w; }
     }
     return acc;
