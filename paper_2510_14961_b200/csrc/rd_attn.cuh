@@ -8,11 +8,14 @@
 // (16-byte cp.async, double buffered) and are reused by every query of the group, so the KV
 // prefix is read once per (sequence, head) for the whole wavefront.  Each warp owns 16 queries:
 // S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with an online
-// softmax in fp32; P is rounded to bf16 for the second product.  Splits write (m, l, O) partials
-// that a second kernel merges in split order (deterministic).
+// softmax in fp32; P is rounded to bf16 for the second product.  The KV splits of one (group, head)
+// form a thread-block cluster: each leaves its (m, l, O) partials in its own shared memory, and
+// after a cluster barrier every block merges the partials of its share of the queries, in split
+// order (deterministic), reading the other blocks' shared memory directly.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <cooperative_groups.h>
 #include <stdint.h>
 
 #include "rd_common.cuh"
@@ -21,7 +24,7 @@ namespace rd {
 
 constexpr int ATT_KT = 64;          // keys per tile
 constexpr int ATT_QMAX = 64;        // queries per group
-constexpr int ATT_MAX_SPLITS = 16;
+constexpr int ATT_MAX_SPLITS = 8;    // = portable cluster size
 
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
     const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
@@ -56,15 +59,13 @@ template <int D> struct AttCfg {
     static constexpr int SMEM = (ATT_QMAX * LD + 4 * ATT_KT * LD) * 2 + ATT_QMAX * 4;
 };
 
-// part_o: [row][head][split][D] unnormalised outputs; part_ml: [row][head][split][2] = (max, sum),
-// the max in the log2 domain of the scaled scores.
+// Grid (splits, heads, groups), clusters of `splits` blocks along x.  out: [rows, hidden] bf16.
 template <int D>
 __global__ void __launch_bounds__(128)
 attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
                    const int* __restrict__ row_seq, int rows_per_group, int n_rows,
                    const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
-                   int hidden, float scale_log2, int n_splits, float* __restrict__ part_o,
-                   float* __restrict__ part_ml) {
+                   int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
     constexpr int LD = AttCfg<D>::LD;
     constexpr int CH = D / 8;           // 16-byte chunks per row
     extern __shared__ __align__(16) uint8_t att_smem[];
@@ -75,8 +76,8 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
 
     pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int hd = blockIdx.x, H = gridDim.x, sp = blockIdx.z;
-    const int r0 = blockIdx.y * rows_per_group;
+    const int sp = blockIdx.x, n_splits = gridDim.x, hd = blockIdx.y;
+    const int r0 = blockIdx.z * rows_per_group;
     const int nq = min(rows_per_group, n_rows - r0);
     if (tid < ATT_QMAX) pos_s[tid] = tid < nq ? row_pos[r0 + tid] : -1;
     __syncthreads();
@@ -193,6 +194,10 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
         }
         __syncthreads();                                   // buffer may be refilled next round
     }
+    // ---- partials to shared memory (the K/V buffers are free now), merge across the cluster ----
+    float* Os = reinterpret_cast<float*>(att_smem);          // [ATT_QMAX][D] unnormalised outputs
+    float* MLs = Os + ATT_QMAX * D;                           // [ATT_QMAX][2] (max in the log2 domain, sum)
+    __syncthreads();
     if (active) {
         // row sums live spread over the quad
         l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
@@ -202,65 +207,53 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
 #pragma unroll
         for (int half = 0; half < 2; half++) {
             const int q = half ? qb : qa;
-            if (q < nq) {
-                const size_t base = ((size_t)(r0 + q) * H + hd) * n_splits + sp;
-                float* po = part_o + base * D;
+            float* po = Os + q * D;
 #pragma unroll
-                for (int j = 0; j < D / 8; j++)
-                    *reinterpret_cast<float2*>(po + j * 8 + 2 * tq) = make_float2(o[j][half * 2], o[j][half * 2 + 1]);
-                if (tq == 0) {
-                    part_ml[base * 2] = half ? m_b : m_a;
-                    part_ml[base * 2 + 1] = half ? l_b : l_a;
-                }
+            for (int j = 0; j < D / 8; j++)
+                *reinterpret_cast<float2*>(po + j * 8 + 2 * tq) = make_float2(o[j][half * 2], o[j][half * 2 + 1]);
+            if (tq == 0) {
+                MLs[q * 2] = half ? m_b : m_a;
+                MLs[q * 2 + 1] = half ? l_b : l_a;
             }
         }
     }
-}
-
-// out[row, head*D + e] = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), splits in ascending order.
-// Block = (row, group of 4 heads), one thread per 4 output elements; the (max, sum) pairs and the
-// partial outputs of all splits are requested before any is used.
-template <int D>
-__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_splits,
-                                    const int* __restrict__ row_pos, int hidden, int n_heads,
-                                    __nv_bfloat16* __restrict__ out) {
-    pdl_enter();
-    constexpr int Q = D / 4;
-    const int r = blockIdx.x;
-    const int hd = blockIdx.y * 4 + threadIdx.x / Q, e = (threadIdx.x % Q) * 4;
-    if (hd >= n_heads) return;
-    __nv_bfloat16* dst = out + (size_t)r * hidden + hd * D + e;
-    if (row_pos[r] < 0) {
-        dst[0] = dst[1] = dst[2] = dst[3] = __float2bfloat16_rn(0.f);
-        return;
-    }
-    const size_t base = ((size_t)r * n_heads + hd) * n_splits;
-    float2 ml[ATT_MAX_SPLITS];
-    float4 o[ATT_MAX_SPLITS];
+    cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+    cluster.sync();
+    // block `sp` merges queries sp, sp + n_splits, ...; one thread per 4 output elements
+    constexpr int Q4 = D / 4;
+    const int mine = nq > sp ? (nq - sp + n_splits - 1) / n_splits : 0;
+    for (int item = tid; item < mine * Q4; item += 128) {
+        const int q = sp + (item / Q4) * n_splits, e = (item % Q4) * 4;
+        __nv_bfloat16* dst = out + (size_t)(r0 + q) * hidden + hd * D + e;
+        float2 ml[ATT_MAX_SPLITS];
+        float4 po[ATT_MAX_SPLITS];
 #pragma unroll
-    for (int s = 0; s < ATT_MAX_SPLITS; s++) {
-        const int ss = min(s, n_splits - 1);
-        ml[s] = __ldcg(reinterpret_cast<const float2*>(part_ml + (base + ss) * 2));
-        o[s] = __ldcg(reinterpret_cast<const float4*>(part_o + (base + ss) * D + e));
-    }
-    float M = -INFINITY;
+        for (int s2 = 0; s2 < ATT_MAX_SPLITS; s2++) {
+            if (s2 < n_splits) {
+                ml[s2] = *reinterpret_cast<const float2*>(cluster.map_shared_rank(MLs, s2) + q * 2);
+                po[s2] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(Os, s2) + q * D + e);
+            }
+        }
+        float M = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < ATT_MAX_SPLITS; s++)
-        if (s < n_splits) M = fmaxf(M, ml[s].x);
-    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-    float den = 0.f;
+        for (int s2 = 0; s2 < ATT_MAX_SPLITS; s2++)
+            if (s2 < n_splits) M = fmaxf(M, ml[s2].x);
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.f;
 #pragma unroll
-    for (int s = 0; s < ATT_MAX_SPLITS; s++) {
-        if (s >= n_splits || ml[s].x == -INFINITY) continue;
-        const float w = exp2f(ml[s].x - M);
-        num.x += o[s].x * w; num.y += o[s].y * w; num.z += o[s].z * w; num.w += o[s].w * w;
-        den += ml[s].y * w;
+        for (int s2 = 0; s2 < ATT_MAX_SPLITS; s2++) {
+            if (s2 >= n_splits || ml[s2].x == -INFINITY) continue;
+            const float w = exp2f(ml[s2].x - M);
+            num.x += po[s2].x * w; num.y += po[s2].y * w; num.z += po[s2].z * w; num.w += po[s2].w * w;
+            den += ml[s2].y * w;
+        }
+        const float inv = (pos_s[q] >= 0 && den > 0.f) ? 1.0f / den : 0.f;     // unused slot: zeros
+        dst[0] = __float2bfloat16_rn(num.x * inv);
+        dst[1] = __float2bfloat16_rn(num.y * inv);
+        dst[2] = __float2bfloat16_rn(num.z * inv);
+        dst[3] = __float2bfloat16_rn(num.w * inv);
     }
-    const float inv = den > 0.f ? 1.0f / den : 0.f;
-    dst[0] = __float2bfloat16_rn(num.x * inv);
-    dst[1] = __float2bfloat16_rn(num.y * inv);
-    dst[2] = __float2bfloat16_rn(num.z * inv);
-    dst[3] = __float2bfloat16_rn(num.w * inv);
+    cluster.sync();                                           // shared memory stays until everyone has read it
 }
 
 }  // namespace rd

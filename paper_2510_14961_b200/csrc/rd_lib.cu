@@ -241,7 +241,6 @@ struct rd_session {
     float* acc = nullptr;          // output of the plain GEMM kernel, [rows, n_out]
     size_t acc_elems = 0;
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
-    float *att_o = nullptr, *att_ml = nullptr;   // split-KV partials of the windowed attention
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
     int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128)
@@ -317,9 +316,6 @@ static void want_max_carveout_everywhere() {
     want_max_carveout(attn_window_kernel<64>);
     want_max_carveout(attn_window_kernel<96>);
     want_max_carveout(attn_window_kernel<128>);
-    want_max_carveout(attn_combine_kernel<64>);
-    want_max_carveout(attn_combine_kernel<96>);
-    want_max_carveout(attn_combine_kernel<128>);
     cudaGetLastError();   // an attribute a kernel does not take is not an error of the session
 }
 
@@ -401,8 +397,6 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if (e == cudaSuccess) e = cudaMemcpy(s->done, ones.data(), B * sizeof(int), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { rc = cuda_fail(e, "session init copies", __LINE__); break; }
         if (c.dtype == RD_BF16 && (c.head_dim == 64 || c.head_dim == 96 || c.head_dim == 128)) {
-            if ((rc = s->mem.get(&s->att_o, R * c.n_heads * ATT_MAX_SPLITS * (size_t)c.head_dim * sizeof(float)))) break;
-            if ((rc = s->mem.get(&s->att_ml, R * c.n_heads * ATT_MAX_SPLITS * 2 * sizeof(float)))) break;
             s->attn_path = 1;
         }
         if (m->tc_ok) {
@@ -545,11 +539,9 @@ template <typename T> struct Eng {
         int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
         ns = std::max(1, std::min(std::min(ns, 8), tiles));
         const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
-        LAUNCH(s, attn_window_kernel<D>, dim3(c.n_heads, groups, ns), 128, AttCfg<D>::SMEM, (const bf16*)s->q_t,
-               s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden, scale_log2, ns, s->att_o,
-               s->att_ml);
-        LAUNCH(s, attn_combine_kernel<D>, dim3(n_rows, (c.n_heads + 3) / 4), D, 0, s->att_o, s->att_ml, ns, s->row_pos,
-               c.hidden, c.n_heads, (bf16*)s->act_h);
+        LAUNCH_CLUSTER(s, attn_window_kernel<D>, (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, (const bf16*)s->q_t,
+                       s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden, scale_log2,
+                       (bf16*)s->act_h);
         return RD_OK;
     }
     static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {
