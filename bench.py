@@ -49,6 +49,25 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "3p5b_b1_p512_g256_W32"
 
+# DRAM bytes (read + write) of one average GEMM launch of a step, from the ncu capture summarised in
+# profiles/gemm_tc_kernel_bn32_3p5b_shapes_W32.md (taken on the 1/1/1-layer case with the same GEMM
+# shapes; the head's traffic scaled by vocabulary).  Valid for the kernel as profiled; set to None
+# when the GEMM kernel changes until the counters are taken again.
+NCU_GEMM_TRAFFIC_PER_LAUNCH = {"3p5b_b1_p512_g256_W32": 217.7e6}
+
+
+def max_over_ranks_sum_tokens(total_ms, tokens, dist=None, device=None):
+    """Whole-job aggregation for N independent replicas: the time is the maximum over ranks, the
+    tokens are summed.  With dist None (one process) the inputs come back unchanged."""
+    if dist is None:
+        return float(total_ms), float(tokens)
+    import torch
+    tm = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    tk = torch.tensor([float(tokens)], dtype=torch.float64, device=device)
+    dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+    return float(tm.item()), float(tk.item())
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -211,12 +230,7 @@ def run_ours(args):
         launches0 = (launches0 or 0) + st1["kernel_launches"] - st0["kernel_launches"]
         steps_done += n
     clk = clocks.stop()
-    tm = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    tk = torch.tensor([float(tokens)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-    total_ms_max, tokens_all = float(tm.item()), float(tk.item())
+    total_ms_max, tokens_all = max_over_ranks_sum_tokens(total_ms, tokens, dist if world > 1 else None, dev)
     df_tok_s = tokens_all / (total_ms_max / 1e3)
     ms_per_step = total_ms_max / K
 
@@ -271,6 +285,8 @@ def run_ours(args):
     barrier()
     t0 = time.perf_counter()
     prefill(e2e)                                            # H2D of the prompts + prefill
+    e2e.sync()
+    e2e_prefill_s = time.perf_counter() - t0
     n_steps_e2e, d2h = 0, 0
     while True:
         e2e.df_step(W, wl["inner"], wl["eps"])
@@ -289,10 +305,8 @@ def run_ours(args):
         d2h += 4 * len(t)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_tok_s = world * got / float(te.item())
+    e2e_s_max, got_all = max_over_ranks_sum_tokens(e2e_s, got, dist if world > 1 else None, dev)
+    e2e_tok_s = got_all / e2e_s_max
     e2e.close()
 
     line = {
@@ -314,7 +328,7 @@ def run_ours(args):
                           "peak_source": peaks["source"]},
         "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections of the step)",
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": NCU_GEMM_TRAFFIC_PER_LAUNCH.get(args.workload),
                      "launches": prof["gemm_launches"], "avg_us": 1e3 * prof["gemm_ms"] / max(prof["gemm_launches"], 1),
                      "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
                      "peak_source": peaks["source"]},
@@ -323,7 +337,8 @@ def run_ours(args):
         "gemm_share_of_step": prof["gemm_ms"] / (prof_steps * ms_per_step) if ms_per_step else None,
         "clocks": clk,
         "e2e": {"value": e2e_tok_s, "unit": "tok/s", "h2d_bytes_per_step": 4.0 * L * B / n_steps_e2e,
-                "d2h_bytes_per_step": d2h / n_steps_e2e, "steps": n_steps_e2e, "includes": "prompt upload, prefill, decode, per-step commit readback, token readback"},
+                "d2h_bytes_per_step": d2h / n_steps_e2e, "steps": n_steps_e2e, "prefill_s": e2e_prefill_s,
+                "total_s": e2e_s, "includes": "prompt upload, prefill, decode, per-step commit readback, token readback"},
         "gpu_launches": int(launches0), "tc_gemm_launches": int(tc_launches),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -34,9 +34,14 @@ class LockStep:
     from the same y_current.  The fp32 configuration uses tie_gap = 0: any mismatch fails."""
 
     def __init__(self, sampler: orc.Sampler, session: rd.Session, seqs, tol: Tolerance, tie_gap=0.0,
-                 check_logits=True):
+                 check_logits=True, logit_noise=None):
+        """logit_noise = (rms, fraction, max_abs): instead of bounding every logit by `tol`, bound the
+        rms error, the fraction of logits outside `tol` and the largest error (used at the full
+        3.5B widths, where bf16 rounding noise amplified by the random-init layers puts a few
+        percent of the 65536 logits per row outside the element-wise bound)."""
         self.sm, self.sess, self.seqs, self.tol, self.tie_gap = sampler, session, seqs, tol, tie_gap
         self.check_logits = check_logits
+        self.logit_noise = logit_noise
         self.near_ties = 0
         self.n_drafts = 0
         self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0}
@@ -65,8 +70,15 @@ class LockStep:
             if self.check_logits:
                 lg = self.sess.debug_read(rd.RD_DBG_LOGITS, b)
                 self.max_err["logits"] = max(self.max_err["logits"], float(np.abs(lg - info["logits"]).max()))
-                assert self.tol.excess(lg, info["logits"]) <= 0, \
-                    f"step {self.steps} seq {b}: logits off by {np.abs(lg - info['logits']).max():.3e}"
+                if self.logit_noise is None:
+                    assert self.tol.excess(lg, info["logits"]) <= 0, \
+                        f"step {self.steps} seq {b}: logits off by {np.abs(lg - info['logits']).max():.3e}"
+                elif lg.size:
+                    err = np.abs(lg - info["logits"])
+                    rms = float(np.sqrt(np.mean(err ** 2)))
+                    frac = float(np.mean(err > self.tol.abs_tol + self.tol.rel_tol * np.abs(info["logits"])))
+                    assert rms <= self.logit_noise[0] and frac <= self.logit_noise[1] and err.max() <= self.logit_noise[2], \
+                        f"step {self.steps} seq {b}: logits rms err {rms:.3e}, outside tolerance {frac:.3%}, max {err.max():.3e}"
             if delta_checked and "delta" in info:
                 dl = self.sess.debug_read(rd.RD_DBG_DELTA, b)
                 fin = np.isfinite(info["delta"])
