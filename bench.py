@@ -39,8 +39,15 @@ WORKLOADS = {
                                  eps=0.0, ar_r=8, prefill_r=8, temperature=0.0),
     "twin_b1_p512_g256_W32": dict(shape=rd_inputs.TWIN, bf16=True, batch=1, prompt=512, gen=256, window=32,
                                   inner=1, eps=0.0, ar_r=32, prefill_r=32, temperature=0.0),
+    # long context (prefill is outside `value`; its recurrence is kept short so that a run stays short)
     "3p5b_b4_p8192_g1024_W32": dict(shape=rd_inputs.SHAPE_3P5B, bf16=True, batch=4, prompt=8192, gen=1024,
-                                    window=32, inner=1, eps=0.0, ar_r=32, prefill_r=32, temperature=0.0),
+                                    window=32, inner=1, eps=0.0, ar_r=32, prefill_r=1, temperature=0.0),
+    # batched serving: 16 sequences, ragged prompts, temperature sampling, adaptive exit
+    "3p5b_b16_ragged_g512_W16": dict(shape=rd_inputs.SHAPE_3P5B, bf16=True, batch=16, prompt=(128, 2048), gen=512,
+                                     window=16, inner=1, eps=1e-3, ar_r=32, prefill_r=1, temperature=1.0),
+    # adaptive exit sweep point (window and inner iterations set on the command line)
+    "3p5b_b1_p1024_g512_adaptive": dict(shape=rd_inputs.SHAPE_3P5B, bf16=True, batch=1, prompt=1024, gen=512,
+                                        window=16, inner=1, eps=1e-3, ar_r=32, prefill_r=4, temperature=0.0),
     # same GEMM and attention shapes as the 3.5B model with 1/1/1 layers and a small vocabulary:
     # about 1.3 GB on the device, for ncu captures
     "3p5b_layers111_v8192_p512_g64_W32": dict(shape=dict(rd_inputs.SHAPE_3P5B, n_prelude=1, n_core=1, n_coda=1, vocab=8192),
@@ -168,7 +175,16 @@ def run_ours(args):
     wl = dict(WORKLOADS[args.workload])
     if args.prefill_r > 0:
         wl["prefill_r"] = args.prefill_r
-    shape, B, L, N, W = wl["shape"], wl["batch"], wl["prompt"], wl["gen"], wl["window"]
+    if args.window > 0:
+        wl["window"] = args.window
+    if args.inner > 0:
+        wl["inner"] = args.inner
+    shape, B, N, W = wl["shape"], wl["batch"], wl["gen"], wl["window"]
+    if isinstance(wl["prompt"], tuple):      # ragged batch: lengths uniform in [lo, hi]
+        lens = [int(x) for x in rd_inputs.make_prompt_lengths(B, wl["prompt"][0], wl["prompt"][1], seed=4)]
+    else:
+        lens = [wl["prompt"]] * B
+    L = max(lens)
     esz = 2 if wl["bf16"] else 4
     peaks = load_peaks()
 
@@ -180,7 +196,7 @@ def run_ours(args):
     torch.cuda.empty_cache()
     stream = torch.cuda.Stream(device=dev)
     max_ctx = L + N + 8
-    prompts = [rd_inputs.make_prompt(L, shape["vocab"], seed=17 + b) for b in range(B)]
+    prompts = [rd_inputs.make_prompt(lens[b], shape["vocab"], seed=17 + b) for b in range(B)]
     pinned = [torch.from_numpy(p).pin_memory() for p in prompts]
 
     def new_session(window, temperature=0.0):
@@ -197,8 +213,6 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    steps_per_gen = N + W - 1 if wl["eps"] <= 0 else None
-    K = args.steps if args.steps > 0 else (steps_per_gen or 300)
     # ---- DF sampler, device-resident ----------------------------------------------------------
     sess = new_session(W, wl["temperature"])
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -209,6 +223,17 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         sess.df_step(W, wl["inner"], wl["eps"])
     sess.sync()
+    if wl["eps"] <= 0:
+        steps_per_gen = N + W - 1            # fixed exit: one token per step after the ramp
+    else:
+        # adaptive exit: the number of steps depends on the latents; an untimed generation with the
+        # same seeds counts them (every run of the same inputs takes the same steps)
+        prefill(sess)
+        steps_per_gen = 0
+        while not all(sess.committed(b)[1] for b in range(B)) and steps_per_gen < 64 * (N + W):
+            sess.df_step(W, wl["inner"], wl["eps"])
+            steps_per_gen += 1
+    K = args.steps if args.steps > 0 else steps_per_gen
     clocks = ClockSampler(local)
     clocks.start()
     total_ms, steps_done, tokens = 0.0, 0, 0
@@ -216,7 +241,7 @@ def run_ours(args):
     while steps_done < K:
         prefill(sess)                       # restart the generation (outside the timed region)
         st0 = sess.stats()
-        n = min(K - steps_done, steps_per_gen or K)
+        n = min(K - steps_done, steps_per_gen)
         barrier()
         with torch.cuda.stream(stream):
             ev0.record(stream)
@@ -249,7 +274,7 @@ def run_ours(args):
     attn_gbs = prof["attn_kv_bytes"] / (prof["attn_ms"] * 1e-3) / 1e9 if prof["attn_ms"] > 0 else 0.0
     tc_launches = sess.stats()["tc_gemm_launches"]
     rows_ss = B * W
-    ctx_mid = B * (L + N // 2)
+    ctx_mid = sum(lens) + B * (N // 2)
     step_b, step_f = step_bytes_flops(shape, B, rows_ss, ctx_mid, wl["inner"], esz)
     t_roof = max(step_b / (peaks["hbm_gbs"] * 1e9), step_f / (peaks["bf16_tflops_sustained"] * 1e12))
     # steady-state step time: the steps profiled above ran with the full window
@@ -271,7 +296,7 @@ def run_ours(args):
     barrier()
     ar_ms = ev0.elapsed_time(ev1)
     ar_tok_s = B * n_ar / (ar_ms / 1e3)
-    ar_b, ar_f = step_bytes_flops(shape, B, B, B * (L + n_ar // 2), wl["ar_r"], esz)
+    ar_b, ar_f = step_bytes_flops(shape, B, B, sum(lens) + B * (n_ar // 2), wl["ar_r"], esz)
     ar_roof = max(ar_b / (peaks["hbm_gbs"] * 1e9), ar_f / (peaks["bf16_tflops_sustained"] * 1e12))
     ar.close()
 
@@ -301,7 +326,7 @@ def run_ours(args):
     got = 0
     for b in range(B):
         t = e2e.tokens(b, out=out_tokens[b].numpy())       # D2H: the generated sequence
-        got += len(t) - L
+        got += len(t) - lens[b]
         d2h += 4 * len(t)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
@@ -314,7 +339,8 @@ def run_ours(args):
         "value": df_tok_s, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl["bf16"] else "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": B, "prompt": L, "generate": N, "window": W,
+        "config": {"workload": args.workload, "batch": B, "prompt": L if len(set(lens)) == 1 else lens, "generate": N, "window": W,
+                   "steps_per_generation": steps_per_gen, "tokens_per_step": tokens_all / (world * K) if K else None,
                    "inner_iters": wl["inner"], "exit_threshold": wl["eps"], "ar_r": wl["ar_r"],
                    "l2": "inputs larger than L2 (weights streamed per step: %.2f GB)" % (step_b / 1e9),
                    "multi_gpu": "replicas only (no data-path collective)"},
@@ -336,7 +362,7 @@ def run_ours(args):
                       "avg_us": 1e3 * prof["attn_ms"] / max(prof["attn_launches"], 1)},
         "gemm_share_of_step": prof["gemm_ms"] / (prof_steps * ms_per_step) if ms_per_step else None,
         "clocks": clk,
-        "e2e": {"value": e2e_tok_s, "unit": "tok/s", "h2d_bytes_per_step": 4.0 * L * B / n_steps_e2e,
+        "e2e": {"value": e2e_tok_s, "unit": "tok/s", "h2d_bytes_per_step": 4.0 * sum(lens) / n_steps_e2e,
                 "d2h_bytes_per_step": d2h / n_steps_e2e, "steps": n_steps_e2e, "prefill_s": e2e_prefill_s,
                 "total_s": e2e_s, "includes": "prompt upload, prefill, decode, per-step commit readback, token readback"},
         "gpu_launches": int(launches0), "tc_gemm_launches": int(tc_launches),
@@ -451,6 +477,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--ar-tokens", type=int, default=24)
+    ap.add_argument("--window", type=int, default=0, help="override the workload's window (sweeps)")
+    ap.add_argument("--inner", type=int, default=0, help="override the workload's inner iterations per step (sweeps)")
     ap.add_argument("--prefill-r", type=int, default=0, help="override the workload's prefill recurrence (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
