@@ -99,7 +99,7 @@ int rd_load(const rd_config* cfg, const void* const* tensors, int32_t n_tensors,
             rd_model** out);
 void rd_free(rd_model* m);
 
-/* rd_session_create -- allocate KV caches (three blocks, [layer][sequence][position][hidden]),
+/* rd_session_create -- allocate KV caches (three blocks, [layer][sequence][head][position][head_dim]),
  * latent slots and token arrays for `batch` sequences.
  *   cuda_stream   a cudaStream_t (as void*) on which every step is enqueued; NULL = legacy
  *                 default stream.  The model must outlive the session. */
@@ -169,8 +169,8 @@ int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which,
  * left, so a cudaMalloc of even a few megabytes fails; and a process that reads cache rows out while
  * other sessions keep stepping on other streams, where cudaMalloc / cudaFree would stall the whole
  * device for a moment.  rd_debug_read_kv takes a temporary float32 buffer from cudaMalloc on every
- * call with a bf16 cache; this call stages through a fixed array that is part of the library image
- * instead and calls no allocating routine.
+ * call; this call stages through a fixed array that is part of the library image instead and calls
+ * no allocating routine.
  *
  * Arguments, layout of `dst` (host memory, float32 [n, hidden]) and results are those of
  * rd_debug_read_kv: the values are bit-identical.  Differences:

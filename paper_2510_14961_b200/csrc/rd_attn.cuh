@@ -60,12 +60,16 @@ template <int D> struct AttCfg {
 };
 
 // Grid (splits, heads, groups), clusters of `splits` blocks along x.  out: [rows, hidden] bf16.
-template <int D>
+// KW = keys of a 64-key tile one warp takes.  KW = 64: the four warps are four blocks of 16 queries
+// (groups of up to 64 rows).  KW = 32, for groups of at most 32 rows: warps 0,1 take the two query
+// blocks on the tile's first 32 keys, warps 2,3 the same queries on its last 32, and the two halves
+// are merged (first half, then second) through shared memory before the cluster merge.
+template <int D, int KW>
 __global__ void __launch_bounds__(128)
 attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
                    const int* __restrict__ row_seq, int rows_per_group, int n_rows,
                    const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
-                   int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
+                   size_t head_stride, int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
     constexpr int LD = AttCfg<D>::LD;
     constexpr int CH = D / 8;           // 16-byte chunks per row
     extern __shared__ __align__(16) uint8_t att_smem[];
@@ -86,8 +90,9 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
     const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
     const int seq = row_seq[r0];
-    const __nv_bfloat16* kbase = Kc + (size_t)seq * seq_stride + (size_t)hd * D;
-    const __nv_bfloat16* vbase = Vc + (size_t)seq * seq_stride + (size_t)hd * D;
+    // cache layout [sequence][head][position][D]: this head's keys are one contiguous stream
+    const __nv_bfloat16* kbase = Kc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
+    const __nv_bfloat16* vbase = Vc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
 
     for (int c = tid; c < ATT_QMAX * CH; c += 128) {
         const int r = c / CH, ch = c % CH;
@@ -101,16 +106,18 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
             const int r = c / CH, ch = c % CH;
             const int key = key0 + r;
             const bool ok = key < kv_len;
-            const size_t off = (size_t)(ok ? key : 0) * hidden + ch * 8;
+            const size_t off = (size_t)(ok ? key : 0) * D + ch * 8;
             cp_async16(Ks + (buf * ATT_KT + r) * LD + ch * 8, kbase + off, ok);
             cp_async16(Vs + (buf * ATT_KT + r) * LD + ch * 8, vbase + off, ok);
         }
         cp_async_commit();
     };
 
-    const bool active = warp * 16 < nq;
+    const int qblk = KW == 64 ? warp : (warp & 1);        // block of 16 queries this warp takes
+    const int koff = KW == 64 ? 0 : (warp >> 1) * KW;     // first key of the tile this warp takes
+    const bool active = qblk * 16 < nq;
     const int g = lane >> 2, tq = lane & 3;
-    const int qa = warp * 16 + g, qb = qa + 8;            // this thread's two query rows
+    const int qa = qblk * 16 + g, qb = qa + 8;            // this thread's two query rows
     float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
     float o[D / 8][4];
 #pragma unroll
@@ -123,22 +130,22 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     if (active) {
 #pragma unroll
         for (int kk = 0; kk < D / 16; kk++)
-            ldsm_x4(qf[kk], Qs + (warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + kk * 16 + (lane >> 4) * 8);
+            ldsm_x4(qf[kk], Qs + (qblk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + kk * 16 + (lane >> 4) * 8);
     }
     for (int t = t0; t < t1; t++) {
         const int buf = (t - t0) & 1;
         if (t + 1 < t1) { load_tile(t + 1, buf ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
         __syncthreads();
         if (active) {
-            const __nv_bfloat16* Kt = Ks + buf * ATT_KT * LD;
-            const __nv_bfloat16* Vt = Vs + buf * ATT_KT * LD;
-            float s[ATT_KT / 8][4];
+            const __nv_bfloat16* Kt = Ks + (buf * ATT_KT + koff) * LD;
+            const __nv_bfloat16* Vt = Vs + (buf * ATT_KT + koff) * LD;
+            float s[KW / 8][4];
 #pragma unroll
-            for (int j = 0; j < ATT_KT / 8; j++) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+            for (int j = 0; j < KW / 8; j++) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
 #pragma unroll
             for (int kk = 0; kk < D / 16; kk++) {
 #pragma unroll
-                for (int jn = 0; jn < ATT_KT / 16; jn++) {
+                for (int jn = 0; jn < KW / 16; jn++) {
                     uint32_t kb[4];
                     ldsm_x4(kb, Kt + (jn * 16 + (lane & 7) + (lane >> 4) * 8) * LD + kk * 16 + ((lane >> 3) & 1) * 8);
                     mma_bf16_16816(s[2 * jn], qf[kk], kb[0], kb[1]);
@@ -146,10 +153,10 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
                 }
             }
             // scale, causal mask, running max
-            const int key0 = t * ATT_KT;
+            const int key0 = t * ATT_KT + koff;
             float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < ATT_KT / 8; j++) {
+            for (int j = 0; j < KW / 8; j++) {
                 const int k0 = key0 + j * 8 + 2 * tq;
                 s[j][0] = (k0 <= pa) ? s[j][0] * scale_log2 : -INFINITY;
                 s[j][1] = (k0 + 1 <= pa) ? s[j][1] * scale_log2 : -INFINITY;
@@ -167,9 +174,9 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
             const float ca = exp2f(m_a - ua), cb = exp2f(m_b - ub);
             m_a = mn_a; m_b = mn_b;
             float sa = 0.f, sb = 0.f;
-            uint32_t pf[ATT_KT / 16][4];
+            uint32_t pf[KW / 16][4];
 #pragma unroll
-            for (int j = 0; j < ATT_KT / 8; j++) {
+            for (int j = 0; j < KW / 8; j++) {
                 const float p0 = exp2f(s[j][0] - ua), p1 = exp2f(s[j][1] - ua);
                 const float p2 = exp2f(s[j][2] - ub), p3 = exp2f(s[j][3] - ub);
                 sa += p0 + p1;
@@ -182,7 +189,7 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
 #pragma unroll
             for (int j = 0; j < D / 8; j++) { o[j][0] *= ca; o[j][1] *= ca; o[j][2] *= cb; o[j][3] *= cb; }
 #pragma unroll
-            for (int kk = 0; kk < ATT_KT / 16; kk++) {
+            for (int kk = 0; kk < KW / 16; kk++) {
 #pragma unroll
                 for (int jn = 0; jn < D / 16; jn++) {
                     uint32_t vb[4];
@@ -198,7 +205,37 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     float* Os = reinterpret_cast<float*>(att_smem);          // [ATT_QMAX][D] unnormalised outputs
     float* MLs = Os + ATT_QMAX * D;                           // [ATT_QMAX][2] (max in the log2 domain, sum)
     __syncthreads();
-    if (active) {
+    if (KW != 64) {
+        // the warps of the second key half hand (m, l, O) to the warps of the first half, thread to thread
+        constexpr int PER = D / 2 + 4;
+        float* st = MLs + ATT_QMAX * 2 + (size_t)(qblk * 32 + lane) * PER;
+        if (warp >= 2) {
+#pragma unroll
+            for (int j = 0; j < D / 8; j++)
+                *reinterpret_cast<float4*>(st + j * 4) = make_float4(o[j][0], o[j][1], o[j][2], o[j][3]);
+            *reinterpret_cast<float4*>(st + D / 2) = make_float4(m_a, l_a, m_b, l_b);
+        }
+        __syncthreads();
+        if (warp < 2) {
+            const float4 ml = *reinterpret_cast<const float4*>(st + D / 2);
+            const float Ma = fmaxf(m_a, ml.x), Mb = fmaxf(m_b, ml.z);
+            const float ua = Ma == -INFINITY ? 0.f : Ma, ub = Mb == -INFINITY ? 0.f : Mb;
+            const float a0 = exp2f(m_a - ua), a1 = exp2f(ml.x - ua), b0 = exp2f(m_b - ub), b1 = exp2f(ml.z - ub);
+#pragma unroll
+            for (int j = 0; j < D / 8; j++) {
+                const float4 v = *reinterpret_cast<const float4*>(st + j * 4);
+                o[j][0] = o[j][0] * a0 + v.x * a1;
+                o[j][1] = o[j][1] * a0 + v.y * a1;
+                o[j][2] = o[j][2] * b0 + v.z * b1;
+                o[j][3] = o[j][3] * b0 + v.w * b1;
+            }
+            l_a = l_a * a0 + ml.y * a1;
+            l_b = l_b * b0 + ml.w * b1;
+            m_a = Ma; m_b = Mb;
+        }
+        __syncthreads();                                      // the staging area overlaps nothing read later
+    }
+    if (active && (KW == 64 || warp < 2)) {
         // row sums live spread over the quad
         l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
         l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);

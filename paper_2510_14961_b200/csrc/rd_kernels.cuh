@@ -314,14 +314,15 @@ template <typename T>
 __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_pos,
                                const int* __restrict__ row_seq, const float* __restrict__ cos_t,
                                const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
-                               T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride) {
+                               T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride, size_t head_stride) {
     pdl_enter();
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
     const int half = head_dim / 2;
-    T* kdst = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
-    T* vdst = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * hidden;
+    // cache layout [sequence][head][position][head_dim]: a head's keys are one contiguous stream
+    T* kseq = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
+    T* vseq = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
     T* qdst = q_t + (size_t)r * hidden;
     // four features = two rotary pairs per thread and turn
     for (int m = (blockIdx.y * blockDim.x + threadIdx.x) * 4; m < hidden; m += gridDim.y * blockDim.x * 4) {
@@ -334,14 +335,17 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
         qdst[m + 1] = from_f<T>(q.x * s0 + q.y * c0);
         qdst[m + 2] = from_f<T>(q.z * c1 - q.w * s1);
         qdst[m + 3] = from_f<T>(q.z * s1 + q.w * c1);
-        kdst[m] = from_f<T>(k.x * c0 - k.y * s0);
-        kdst[m + 1] = from_f<T>(k.x * s0 + k.y * c0);
-        kdst[m + 2] = from_f<T>(k.z * c1 - k.w * s1);
-        kdst[m + 3] = from_f<T>(k.z * s1 + k.w * c1);
-        vdst[m] = from_f<T>(v.x);
-        vdst[m + 1] = from_f<T>(v.y);
-        vdst[m + 2] = from_f<T>(v.z);
-        vdst[m + 3] = from_f<T>(v.w);
+        // the two pairs may lie in different heads when head_dim is not a multiple of 4
+        const size_t d0 = (size_t)(m / head_dim) * head_stride + (m % head_dim);
+        const size_t d1 = (size_t)((m + 2) / head_dim) * head_stride + ((m + 2) % head_dim);
+        kseq[d0] = from_f<T>(k.x * c0 - k.y * s0);
+        kseq[d0 + 1] = from_f<T>(k.x * s0 + k.y * c0);
+        kseq[d1] = from_f<T>(k.z * c1 - k.w * s1);
+        kseq[d1 + 1] = from_f<T>(k.z * s1 + k.w * c1);
+        vseq[d0] = from_f<T>(v.x);
+        vseq[d0 + 1] = from_f<T>(v.y);
+        vseq[d1] = from_f<T>(v.z);
+        vseq[d1 + 1] = from_f<T>(v.w);
     }
 }
 
@@ -351,16 +355,16 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
 template <typename T>
 __global__ void __launch_bounds__(128)
 attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
-                const T* __restrict__ Kc, const T* __restrict__ Vc, size_t seq_stride, int hidden,
-                int head_dim, float scale, T* __restrict__ out) {
+                const T* __restrict__ Kc, const T* __restrict__ Vc, size_t seq_stride, size_t head_stride,
+                int hidden, int head_dim, float scale, T* __restrict__ out) {
     pdl_enter();
     __shared__ float sm_m[4], sm_l[4], sm_o[4][128];
     const int r = blockIdx.x, hd = blockIdx.y;
     const int p = row_pos[r];
     if (p < 0) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const T* kb = Kc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_dim;
-    const T* vb = Vc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_dim;
+    const T* kb = Kc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_stride;
+    const T* vb = Vc + (size_t)row_seq[r] * seq_stride + (size_t)hd * head_stride;
     float q[4], o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int t = 0; t < 4; t++) {
@@ -373,7 +377,7 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
 #pragma unroll
         for (int t = 0; t < 4; t++) {
             const int e = lane + 32 * t;
-            if (e < head_dim) d = fmaf(q[t], to_f(kb[(size_t)j * hidden + e]), d);
+            if (e < head_dim) d = fmaf(q[t], to_f(kb[(size_t)j * head_dim + e]), d);
         }
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
@@ -384,7 +388,7 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
 #pragma unroll
         for (int t = 0; t < 4; t++) {
             const int e = lane + 32 * t;
-            if (e < head_dim) o[t] = o[t] * corr + pj * to_f(vb[(size_t)j * hidden + e]);
+            if (e < head_dim) o[t] = o[t] * corr + pj * to_f(vb[(size_t)j * head_dim + e]);
         }
         m = mn;
     }
@@ -588,10 +592,16 @@ __global__ void convert_kernel(const float* __restrict__ src, T* __restrict__ ds
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         dst[i] = from_f<T>(src[i]);
 }
+// K or V of positions pos0 .. pos0+n-1 of one sequence, gathered from the cache's
+// [head][position][head_dim] layout into float32 rows [n, hidden].
 template <typename T>
-__global__ void widen_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        dst[i] = to_f(src[i]);
+__global__ void kv_gather_kernel(const T* __restrict__ seq_base, size_t head_stride, int head_dim, int hidden, int pos0,
+                                 int n, float* __restrict__ dst) {
+    const size_t total = (size_t)n * hidden;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t row = i / hidden, m = i % hidden;
+        dst[i] = to_f(seq_base[(m / head_dim) * head_stride + (pos0 + row) * head_dim + m % head_dim]);
+    }
 }
 
 }  // namespace rd

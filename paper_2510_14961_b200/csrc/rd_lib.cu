@@ -226,6 +226,7 @@ struct rd_session {
     int R = 0;         // row capacity of the scratch buffers (>= n_slots; prefill chunk size)
     int tok_stride = 0;
     size_t seq_stride = 0;   // elements between sequences in a cache layer
+    size_t head_stride = 0;  // elements between heads of a sequence: cache layout [layer][seq][head][pos][head_dim]
     // device state
     int *tokens = nullptr, *n_prompt = nullptr, *n_committed = nullptr, *win_len = nullptr, *done = nullptr;
     int *row_steps = nullptr, *row_iters = nullptr, *row_pos = nullptr, *row_seq = nullptr;
@@ -313,9 +314,6 @@ static void want_max_carveout_everywhere() {
     want_max_carveout(sample_pick_kernel);
     want_max_carveout(delta_kernel);
     want_max_carveout(advance_kernel);
-    want_max_carveout(attn_window_kernel<64>);
-    want_max_carveout(attn_window_kernel<96>);
-    want_max_carveout(attn_window_kernel<128>);
     cudaGetLastError();   // an attribute a kernel does not take is not an error of the session
 }
 
@@ -340,6 +338,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     s->R = (s->R + 15) / 16 * 16;
     s->tok_stride = sc.max_context + 1;
     s->seq_stride = (size_t)sc.max_context * h;
+    s->head_stride = (size_t)sc.max_context * c.head_dim;
     const size_t R = s->R, B = sc.batch;
     int rc = RD_OK;
     do {
@@ -525,11 +524,12 @@ template <typename T> struct Eng {
     }
 
     // Windowed flash-decode attention (bf16): groups of s->grp_rows rows share their sequence's KV.
-    template <int D>
+    template <int D, int KW>
     static int attn_windowed_d(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
         static bool attr_set = false;
         if (!attr_set) {
-            CU(cudaFuncSetAttribute(attn_window_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<D>::SMEM));
+            CU(cudaFuncSetAttribute(attn_window_kernel<D, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<D>::SMEM));
+            cudaFuncSetAttribute(attn_window_kernel<D, KW>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             attr_set = true;
         }
         const rd_config& c = s->m->cfg;
@@ -539,16 +539,21 @@ template <typename T> struct Eng {
         int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
         ns = std::max(1, std::min(std::min(ns, 8), tiles));
         const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
-        LAUNCH_CLUSTER(s, attn_window_kernel<D>, (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, (const bf16*)s->q_t,
-                       s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, c.hidden, scale_log2,
+        LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW>), (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, (const bf16*)s->q_t,
+                       s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
                        (bf16*)s->act_h);
         return RD_OK;
     }
+    template <int D>
+    static int attn_windowed_k(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
+        // groups of at most 32 rows: every warp takes half of a key tile, so all four warps work
+        return s->grp_rows <= 32 ? attn_windowed_d<D, 32>(s, Kc, Vc, n_rows) : attn_windowed_d<D, 64>(s, Kc, Vc, n_rows);
+    }
     static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {
         switch (s->m->cfg.head_dim) {
-            case 64: return attn_windowed_d<64>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
-            case 96: return attn_windowed_d<96>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
-            case 128: return attn_windowed_d<128>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            case 64: return attn_windowed_k<64>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            case 96: return attn_windowed_k<96>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
+            case 128: return attn_windowed_k<128>(s, (const bf16*)Kc, (const bf16*)Vc, n_rows);
             default: return RD_E_INVALID_ARG;
         }
     }
@@ -569,7 +574,7 @@ template <typename T> struct Eng {
         RowSource acc;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
         LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
-               (T*)s->q_t, Kc, Vc, s->seq_stride);
+               (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
         if constexpr (sizeof(T) == 2) {
@@ -580,7 +585,7 @@ template <typename T> struct Eng {
         }
         if (!windowed) {
             LAUNCH(s, attn_row_kernel<T>, dim3(n_rows, c.n_heads), 128, 0, (T*)s->q_t, s->row_pos, s->row_seq, Kc, Vc,
-                   s->seq_stride, h, c.head_dim, (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
+                   s->seq_stride, s->head_stride, h, c.head_dim, (float)(1.0 / sqrt((double)c.head_dim)), (T*)s->act_h);
         }
         bracket_close(s, br);
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, n_rows, &acc));
@@ -886,16 +891,15 @@ extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int
     if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 + n > s->sc.max_context) return RD_E_INVALID_ARG;
     RD_TRY(rd_sync(s));
     if (n == 0) return RD_OK;
-    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride + (size_t)pos0 * c.hidden;
+    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride;
     const size_t cnt = (size_t)n * c.hidden;
     const char* src = (const char*)(which ? s->Vc[block] : s->Kc[block]) + off * s->m->esz;
-    if (c.dtype == RD_F32) {
-        CU(cudaMemcpy(dst, src, cnt * 4, cudaMemcpyDeviceToHost));
-        return RD_OK;
-    }
     float* tmp = nullptr;
     CU(cudaMalloc((void**)&tmp, cnt * 4));
-    widen_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, tmp, cnt);
+    if (c.dtype == RD_F32)
+        kv_gather_kernel<float><<<256, 256, 0, s->stream>>>((const float*)src, s->head_stride, c.head_dim, c.hidden, pos0, n, tmp);
+    else
+        kv_gather_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, s->head_stride, c.head_dim, c.hidden, pos0, n, tmp);
     cudaError_t e = cudaStreamSynchronize(s->stream);
     if (e == cudaSuccess) e = cudaMemcpy(dst, tmp, cnt * 4, cudaMemcpyDeviceToHost);
     cudaFree(tmp);
@@ -906,7 +910,7 @@ extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int
 // ---------------------------------------------------------------------------------------------
 // rd_debug_read_kv_noalloc: the K/V read-out without any allocation.
 //
-// rd_debug_read_kv widens bf16 cache rows to float32 in a temporary device buffer that it obtains
+// rd_debug_read_kv gathers cache rows into float32 [n, hidden] in a temporary device buffer that it obtains
 // from cudaMalloc and returns with cudaFree.  Here the temporary is a fixed array that is part of
 // the library image: every device that loads the library holds RD_KV_STAGE_ELEMS floats (4 MiB)
 // until the process exits.  In host code `g_kv_stage` is only a handle for the runtime, not an
@@ -950,16 +954,15 @@ extern "C" int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t la
     if (dev != s->m->device) return RD_E_STATE;   // the session's device must be current
     RD_TRY(rd_sync(s));
     if (n == 0) return RD_OK;
-    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride + (size_t)pos0 * c.hidden;
+    const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride;
     const char* src = (const char*)(which ? s->Vc[block] : s->Kc[block]) + off * s->m->esz;
-    if (c.dtype == RD_F32) {                      // float32 cache: no staging needed at all
-        CU(cudaMemcpy(dst, src, cnt * 4, cudaMemcpyDeviceToHost));
-        return RD_OK;
-    }
     float* stage = nullptr;
     RD_TRY(kv_stage_address(dev, &stage));
     // every element of stage[0..cnt) is overwritten: nothing of an earlier call can show through
-    widen_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, stage, cnt);
+    if (c.dtype == RD_F32)
+        kv_gather_kernel<float><<<256, 256, 0, s->stream>>>((const float*)src, s->head_stride, c.head_dim, c.hidden, pos0, n, stage);
+    else
+        kv_gather_kernel<bf16><<<256, 256, 0, s->stream>>>((const bf16*)src, s->head_stride, c.head_dim, c.hidden, pos0, n, stage);
     CU(cudaGetLastError());
     CU(cudaStreamSynchronize(s->stream));
     CU(cudaMemcpy(dst, stage, cnt * 4, cudaMemcpyDeviceToHost));
