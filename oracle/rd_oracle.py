@@ -18,6 +18,8 @@ What follows the paper and where:
 * autoregressive sampler -- Section 3.1 display applied token by token.
 * diffusion-forcing sampler, fixed exit -- Algorithm 1; adaptive exit --
   Eq. 3 (delta_i and k*) and Algorithm 2; wavefront limiter -- Section 3.5.
+* stabilisers: momentum on the conditioning and scheduled latent noise --
+  Section 3.4 (both displays), Algorithm 1 lines 6-7.
 
 The paper does not print the layer internals; the reading used here (pre-norm
 residual layers, RMSNorm, rotary embedding on adjacent pairs, SwiGLU, one
@@ -56,6 +58,7 @@ _SH32 = np.uint64(32)
 
 STREAM_INIT_STATE = 0
 STREAM_GUMBEL = 1
+STREAM_NOISE = 2
 
 
 def philox4x32_10(ctr, key):
@@ -100,6 +103,21 @@ def init_state(seed, seq, pos, hidden, sigma, dtype):
     """
     nb = (hidden + 3) // 4
     u = _unit_interval(_draw_blocks(seed, STREAM_INIT_STATE, seq, pos, nb))
+    out = np.empty((nb, 4), dtype=np.float64)
+    for a in (0, 2):
+        r = np.sqrt(-2.0 * np.log(u[:, a]))
+        th = 2.0 * math.pi * u[:, a + 1]
+        out[:, a] = r * np.cos(th)
+        out[:, a + 1] = r * np.sin(th)
+    return (sigma * out.reshape(-1)[:hidden]).astype(dtype)
+
+
+def latent_noise(seed, seq, pos, step, hidden, sigma, dtype):
+    """z_noise of the noise-injection stabiliser (Section 3.4, second display): a fresh N(0, sigma^2 I)
+    draw for position `pos` at its `step`-th sampler step.  Same construction as init_state on the
+    noise stream; the step index sits in bits 8.. of the counter's stream word."""
+    nb = (hidden + 3) // 4
+    u = _unit_interval(_draw_blocks(seed, STREAM_NOISE | (int(step) << 8), seq, pos, nb))
     out = np.empty((nb, 4), dtype=np.float64)
     for a in (0, 2):
         r = np.sqrt(-2.0 * np.log(u[:, a]))
@@ -278,6 +296,7 @@ class Row:
     z: np.ndarray
     steps: int = 0      # sampler steps this position has taken
     iters: int = 0      # core iterations this position has taken (steps * r')
+    e_prev: object = None   # input conditioning e this position used in the previous step (momentum)
 
 
 @dataclass
@@ -298,11 +317,18 @@ class Sequence:
 
 
 class Sampler:
-    def __init__(self, model: RDModel, seed=0, temperature=0.0, max_iters_per_pos=64):
+    def __init__(self, model: RDModel, seed=0, temperature=0.0, max_iters_per_pos=64, eta=0.0, beta=0.0):
+        """eta: momentum on the input conditioning, e = eta e_prev + (1 - eta) P(y_current)
+        (Section 3.4, first display); a position's first step has no e_prev and takes P(.) as is.
+        beta: latent noise, z' = (1 - beta_t) z + beta_t z_noise (second display), beta_t falling
+        linearly with the steps t a position has taken: beta_t = beta max(0, 1 - t / T), T the
+        number of steps a position gets (the window when the exit is fixed, cap / r' otherwise)."""
         self.m = model
         self.seed = seed
         self.temperature = temperature
         self.cap = max_iters_per_pos
+        self.eta = eta
+        self.beta = beta
 
     def _init(self, seq_id, pos):
         c = self.m.cfg
@@ -367,8 +393,22 @@ class Sampler:
         # e <- P(y_current): the oldest row reads the last committed token, the others the
         # drafts of the previous step.
         e = self.m.prelude(sq.tokens[pos], pos, sq.caches)
+        if self.eta > 0.0:                                # momentum on the conditioning
+            e = e.copy()
+            for i, r_ in enumerate(rows):
+                if r_.e_prev is not None:
+                    e[i] = np.float32(self.eta) * r_.e_prev + np.float32(1.0 - self.eta) * e[i]
+                r_.e_prev = e[i].copy()
         z_prev = np.stack([r_.z for r_ in rows])
         z = z_prev
+        if self.beta > 0.0:                               # noise injection, less of it at later steps
+            c = self.m.cfg
+            T = window if exit_threshold <= 0 else -(-self.cap // inner_iters)
+            z = z.copy()
+            for i, r_ in enumerate(rows):
+                bt = np.float32(self.beta * max(0.0, 1.0 - r_.steps / T))
+                noise = latent_noise(self.seed, sq.seq_id, r_.pos, r_.steps, c.hidden, c.init_sigma, self.m.dtype)
+                z[i] = (np.float32(1.0) - bt) * z[i] + bt * noise
         for _ in range(inner_iters):                      # inner recurrence
             z = self.m.core(e, z, pos, sq.caches)
         logits = self.m.coda(z, pos, sq.caches)           # every in-flight row yields a draft
