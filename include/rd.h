@@ -71,7 +71,14 @@ typedef struct {
     int32_t keep_logits;       /* non-zero: full logits of the last step stay readable       */
     float temperature;         /* 0 => greedy (arg max, lowest index on ties); else Gumbel-max
                                   sampling from softmax(logits / temperature)                */
-    uint64_t seed;             /* key of the counter-based generator (initial states, Gumbel) */
+    uint64_t seed;             /* key of the counter-based generator (initial states, Gumbel, noise) */
+    float eta;                 /* Section 3.4: momentum on the input conditioning of rd_df_step,
+                                  e = eta e_prev + (1 - eta) P(y_current) from a position's second
+                                  step on; 0 <= eta < 1, 0 = off                                  */
+    float beta;                /* Section 3.4 / Algorithm 1 lines 6-7: latent noise in rd_df_step,
+                                  z <- (1 - b_t) z + b_t z_noise, b_t = beta max(0, 1 - t / T) at a
+                                  position's step t; T = window (fixed exit) or
+                                  ceil(max_iters_per_pos / inner_iters); 0 <= beta <= 1, 0 = off  */
 } rd_session_config;
 
 typedef struct {
@@ -125,8 +132,9 @@ int rd_ar_step(rd_session* s, int32_t r);
  * commit the longest finished prefix, append one fresh position while fewer than `window` rows
  * are in flight.  exit_threshold <= 0: fixed exit (Algorithm 1; a row is finished after `window`
  * steps).  exit_threshold > 0: adaptive exit (Algorithm 2; finished when delta_i of Eq. 3 is below
- * the threshold, or after max_iters_per_pos core iterations).  rd_df_step(1, r, 0) computes exactly
- * what rd_ar_step(r) computes.  Errors: STATE, CAPACITY (window > max_window), INVALID_ARG. */
+ * the threshold, or after max_iters_per_pos core iterations).  With eta = beta = 0,
+ * rd_df_step(1, r, 0) computes exactly what rd_ar_step(r) computes (rd_ar_step never applies the
+ * stabilisers).  Errors: STATE, CAPACITY (window > max_window), INVALID_ARG. */
 int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, float exit_threshold);
 
 /* rd_sync -- wait for every enqueued step; returns TIMEOUT/CUDA if a kernel reported a fault. */

@@ -72,7 +72,7 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
     }
     return c;
 }
-enum { STREAM_INIT_STATE = 0, STREAM_GUMBEL = 1 };
+enum { STREAM_INIT_STATE = 0, STREAM_GUMBEL = 1, STREAM_NOISE = 2 };
 
 // u = ((x >> 9) + 1/2) 2^-23 lies in (0,1) and is exact in float32.
 __device__ __forceinline__ float unit_open(uint32_t x) { return ((float)(x >> 9) + 0.5f) * 1.1920928955078125e-07f; }
@@ -107,45 +107,62 @@ __global__ void fill_rows_kernel(int seq, int start, int n, int n_slots, int* __
     row_seq[i] = seq;
 }
 
-// s_0 ~ N(0, sigma^2 I), keyed by (seed, sequence, position): element j is output j%4 of block
-// j/4; the block's words x0..x3 give two Box-Muller pairs.  Evaluated in double (a few thousand
-// values per new row).  only_fresh: fill rows whose step counter is 0 (rows appended last step).
+// Four N(0, sigma^2) values from one Philox block: two Box-Muller pairs, evaluated in double.
+__device__ __forceinline__ void normal4(uint4 x, float sigma, float* out) {
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int a = 0; a < 4; a += 2) {
+        const double u0 = ((double)(w[a] >> 9) + 0.5) * 1.1920928955078125e-07;
+        const double u1 = ((double)(w[a + 1] >> 9) + 0.5) * 1.1920928955078125e-07;
+        const double rad = sqrt(-2.0 * log(u0));
+        double sn, cs;
+        sincos(6.283185307179586476925286766559 * u1, &sn, &cs);
+        out[a] = (float)((double)sigma * (rad * cs));
+        out[a + 1] = (float)((double)sigma * (rad * sn));
+    }
+}
+
+// Start of a pass over the rows.
+// s_0 ~ N(0, sigma^2 I), keyed by (seed, sequence, position): element j is output j%4 of block j/4.
+// only_fresh: only rows whose step counter is 0 (rows appended last step) get s_0; the others keep z.
 // With z_prev the kernel also takes the snapshot z_prev <- z of every active row (Algorithm 2).
+// With beta > 0 it then mixes noise into z (Section 3.4): z <- (1 - b) z + b z_noise, b = beta
+// max(0, 1 - t / sched_steps) for a row that has taken t steps, z_noise a fresh N(0, sigma^2 I) draw
+// keyed by (seed, sequence, position, t) on its own stream.
 __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                                   const int* __restrict__ row_steps, int only_fresh, int hidden,
                                   float sigma, uint64_t seed, float* __restrict__ z, size_t ldz,
-                                  float* __restrict__ z_prev) {
+                                  float* __restrict__ z_prev, float beta, int sched_steps) {
     pdl_enter();
     const int r = blockIdx.x;
     const int p = row_pos[r];
     if (p < 0) return;
-    if (only_fresh && row_steps[r] != 0) {
-        // a row already in flight: only the snapshot z_prev <- z of the step's start is taken
-        if (z_prev)
-            for (int j = threadIdx.x; j < hidden; j += blockDim.x) z_prev[(size_t)r * ldz + j] = z[(size_t)r * ldz + j];
-        return;
-    }
+    const int t = only_fresh ? row_steps[r] : 0;
+    const bool fresh = !only_fresh || t == 0;
+    const float b = beta > 0.f ? beta * fmaxf(0.f, 1.0f - (float)t / (float)sched_steps) : 0.f;
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint32_t seq = (uint32_t)row_seq[r];
     const int nb = (hidden + 3) / 4;
     for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
-        const uint4 x = philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, (uint32_t)row_seq[r], STREAM_INIT_STATE), key);
-        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-        float out[4];
+        float v[4];
+        if (fresh) {
+            normal4(philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, seq, STREAM_INIT_STATE), key), sigma, v);
+        } else {
 #pragma unroll
-        for (int a = 0; a < 4; a += 2) {
-            const double u0 = ((double)(w[a] >> 9) + 0.5) * 1.1920928955078125e-07;
-            const double u1 = ((double)(w[a + 1] >> 9) + 0.5) * 1.1920928955078125e-07;
-            const double rad = sqrt(-2.0 * log(u0));
-            double sn, cs;
-            sincos(6.283185307179586476925286766559 * u1, &sn, &cs);
-            out[a] = (float)((double)sigma * (rad * cs));
-            out[a + 1] = (float)((double)sigma * (rad * sn));
+            for (int a = 0; a < 4; a++) v[a] = blk * 4 + a < hidden ? z[(size_t)r * ldz + blk * 4 + a] : 0.f;
+        }
+        float zn[4] = {v[0], v[1], v[2], v[3]};
+        if (b > 0.f) {
+            float nz[4];
+            normal4(philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, seq, STREAM_NOISE | ((uint32_t)t << 8)), key), sigma, nz);
+#pragma unroll
+            for (int a = 0; a < 4; a++) zn[a] = __fadd_rn(__fmul_rn(1.0f - b, v[a]), __fmul_rn(b, nz[a]));
         }
 #pragma unroll
         for (int a = 0; a < 4; a++)
             if (blk * 4 + a < hidden) {
-                z[(size_t)r * ldz + blk * 4 + a] = out[a];
-                if (z_prev) z_prev[(size_t)r * ldz + blk * 4 + a] = out[a];
+                if (fresh || b > 0.f) z[(size_t)r * ldz + blk * 4 + a] = zn[a];
+                if (z_prev) z_prev[(size_t)r * ldz + blk * 4 + a] = v[a];
             }
     }
 }
@@ -221,9 +238,11 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
 }
 
 // out[row] = src[row] (+ resid[row]) as a plain float32 array (n multiple of 4: vector path).
+// With eta > 0 (momentum on the input conditioning, Section 3.4) a row that has already taken a step
+// gets out = eta out_old + (1 - eta) (src + resid); a row at its first step has no out_old.
 __global__ void reduce_store_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
                                     float* __restrict__ out, size_t ldo, int n, int n_rows,
-                                    const int* __restrict__ row_pos) {
+                                    const int* __restrict__ row_pos, const int* __restrict__ row_steps, float eta) {
     pdl_enter();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if ((n & 3) == 0) {
@@ -236,15 +255,27 @@ __global__ void reduce_store_kernel(const RowSource src, const float* __restrict
             const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
         }
-        *reinterpret_cast<float4*>(out + (size_t)r * ldo + m) = v;
+        float4* dst = reinterpret_cast<float4*>(out + (size_t)r * ldo + m);
+        if (eta > 0.f && row_steps[r] > 0) {
+            const float4 o = *dst;
+            const float k = 1.0f - eta;
+            v.x = __fadd_rn(__fmul_rn(eta, o.x), __fmul_rn(k, v.x));
+            v.y = __fadd_rn(__fmul_rn(eta, o.y), __fmul_rn(k, v.y));
+            v.z = __fadd_rn(__fmul_rn(eta, o.z), __fmul_rn(k, v.z));
+            v.w = __fadd_rn(__fmul_rn(eta, o.w), __fmul_rn(k, v.w));
+        }
+        *dst = v;
     } else {
         const size_t per_row = ((size_t)n + 3) / 4;
         if (i >= (size_t)n_rows * per_row) return;
         const int r = (int)(i / per_row), m0 = (int)(i % per_row) * 4;
         if (row_pos[r] < 0) return;
+        const bool mix = eta > 0.f && row_steps[r] > 0;
         for (int m = m0; m < min(m0 + 4, n); m++) {
-            const float v = row_source_load(src, r, m);
-            out[(size_t)r * ldo + m] = resid ? resid[(size_t)r * ldr + m] + v : v;
+            float v = row_source_load(src, r, m);
+            if (resid) v += resid[(size_t)r * ldr + m];
+            float* dst = out + (size_t)r * ldo + m;
+            *dst = mix ? __fadd_rn(__fmul_rn(eta, *dst), __fmul_rn(1.0f - eta, v)) : v;
         }
     }
 }

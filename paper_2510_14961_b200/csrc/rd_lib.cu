@@ -323,6 +323,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     const rd_session_config& sc = *scp;
     if (sc.batch < 1 || sc.max_context < 2 || sc.max_window < 1 || sc.max_new_tokens < 0) return RD_E_INVALID_ARG;
     if (sc.max_iters_per_pos < 1 || !(sc.temperature >= 0.f)) return RD_E_INVALID_ARG;
+    if (!(sc.eta >= 0.f && sc.eta < 1.f) || !(sc.beta >= 0.f && sc.beta <= 1.f)) return RD_E_INVALID_ARG;
     if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
     rd_session* s = new (std::nothrow) rd_session();
     if (!s) return RD_E_OOM;
@@ -599,28 +600,28 @@ template <typename T> struct Eng {
         return RD_OK;
     }
 
-    // dst[row] = x[row] for a pending x.
-    static int materialise(rd_session* s, const Pending& in, float* dst, int n, int n_rows) {
+    // dst[row] = x[row] for a pending x; eta > 0: momentum on rows that have taken a step (see the kernel).
+    static int materialise(rd_session* s, const Pending& in, float* dst, int n, int n_rows, float eta = 0.f) {
         const size_t items = (size_t)n_rows * ((n + 3) / 4);
         LAUNCH(s, reduce_store_kernel, (unsigned)((items + 255) / 256), 256, 0, in.src, in.resid, (size_t)n, dst, (size_t)n, n,
-               n_rows, s->row_pos);
+               n_rows, s->row_pos, s->row_steps, eta);
         return RD_OK;
     }
 
-    // e_out = P(tokens of the rows): embedding + prelude layers.
-    static int prelude(rd_session* s, int n_rows, float* e_out) {
+    // e_out = P(tokens of the rows): embedding + prelude layers (eta: momentum, decode steps only).
+    static int prelude(rd_session* s, int n_rows, float* e_out, float eta = 0.f) {
         const rd_config& c = s->m->cfg;
-        float* x0 = c.n_prelude > 0 ? s->x : e_out;
-        LAUNCH(s, embed_kernel<T>, dim3(n_rows, 4), 128, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride, (const T*)s->m->emb,
-               c.hidden, x0);
-        if (c.n_prelude == 0) return RD_OK;
+        const bool via_x = c.n_prelude > 0 || eta > 0.f;
+        LAUNCH(s, embed_kernel<T>, dim3(n_rows, 4), 128, 0, s->row_pos, s->row_seq, s->tokens, s->tok_stride,
+               (const T*)s->m->emb, c.hidden, via_x ? s->x : e_out);
+        if (!via_x) return RD_OK;
         Pending x = plain_rows(s->x, c.hidden);
         for (int l = 0; l < c.n_prelude; l++) {
             Pending y;
             RD_TRY(layer(s, 0, l, x, &y, n_rows));
             x = y;
         }
-        return materialise(s, x, e_out, c.hidden, n_rows);
+        return materialise(s, x, e_out, c.hidden, n_rows, eta);
     }
 
     // z_out = R(e, z_in): adapter over concat(e, z), core layers, closing RMSNorm.
@@ -668,7 +669,7 @@ template <typename T> struct Eng {
     }
 
     // One sampler step over the decode slots (Algorithm 1 / Algorithm 2; AR is window 1).
-    static int decode_step(rd_session* s, int window, int inner, float eps) {
+    static int decode_step(rd_session* s, int window, int inner, float eps, bool stabilise) {
         const rd_config& c = s->m->cfg;
         const int n = s->n_slots, h = c.hidden, B = s->sc.batch;
         // the leading edge of a wavefront advances by at most one position per step
@@ -685,9 +686,12 @@ template <typename T> struct Eng {
         LAUNCH(s, plan_rows_kernel, (n + 127) / 128, 128, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window,
                s->row_pos, s->row_seq, s->step_first, s->step_n);
         // s_0 for the rows appended by the previous step, and the snapshot z_prev <- z
+        // (stabilisers of Section 3.4 apply to sampler steps, not to the sequential decoder)
+        const float eta = stabilise ? s->sc.eta : 0.f, beta = stabilise ? s->sc.beta : 0.f;
+        const int sched = eps <= 0.f ? window : (s->sc.max_iters_per_pos + inner - 1) / inner;
         LAUNCH(s, init_state_kernel, n, 128, 0, s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma, s->sc.seed, s->z,
-               (size_t)h, s->z_prev);
-        RD_TRY(prelude(s, n, s->e));
+               (size_t)h, s->z_prev, beta, sched);
+        RD_TRY(prelude(s, n, s->e, eta));
         for (int j = 0; j < inner; j++) RD_TRY(core(s, s->e, s->z, s->z, n));
         RD_TRY(coda(s, s->z, n, true));
         LAUNCH(s, delta_kernel, n, 256, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
@@ -714,7 +718,7 @@ template <typename T> struct Eng {
                 if (pass == 0) {
                     RD_TRY(prelude(s, nr, ec));
                     LAUNCH(s, init_state_kernel, nr, 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
-                           s->sc.seed, zc, (size_t)h, (float*)nullptr);
+                           s->sc.seed, zc, (size_t)h, (float*)nullptr, 0.f, 1);
                 } else if (pass <= r) {
                     RD_TRY(core(s, ec, zc, zc, nr));
                 } else {
@@ -787,7 +791,7 @@ extern "C" int rd_ar_step(rd_session* s, int32_t r) {
     if (!any_prefilled(s)) return RD_E_STATE;
     for (int b = 0; b < s->sc.batch; b++)
         if (s->prefilled[b] && s->wave_open[b]) return RD_E_STATE;
-    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, 1, r, 0.f) : Eng<float>::decode_step(s, 1, r, 0.f);
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, 1, r, 0.f, false) : Eng<float>::decode_step(s, 1, r, 0.f, false);
     if (rc == RD_OK) s->stats.ar_steps++;
     return rc;
 }
@@ -796,8 +800,8 @@ extern "C" int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, fl
     if (!s || window < 1 || inner_iters < 1 || exit_threshold != exit_threshold) return RD_E_INVALID_ARG;
     if (window > s->sc.max_window) return RD_E_CAPACITY;
     if (!any_prefilled(s)) return RD_E_STATE;
-    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, window, inner_iters, exit_threshold)
-                                              : Eng<float>::decode_step(s, window, inner_iters, exit_threshold);
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, window, inner_iters, exit_threshold, true)
+                                              : Eng<float>::decode_step(s, window, inner_iters, exit_threshold, true);
     if (rc == RD_OK) {
         s->stats.df_steps++;
         if (window > 1)
