@@ -216,6 +216,8 @@ def run_ours(args):
     # ---- DF sampler, device-resident ----------------------------------------------------------
     sess = new_session(W, wl["temperature"])
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    prefill(sess)                            # first call: also loads the kernels
+    sess.sync()
     t_pf0 = time.perf_counter()
     prefill(sess)
     sess.sync()

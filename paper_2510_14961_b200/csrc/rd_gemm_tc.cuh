@@ -9,7 +9,8 @@
 // (128 lanes x BN columns, fp32, two buffers).
 //
 // Persistent stream-K schedule: the (feature tile, row tile, k-block) units are numbered tile by
-// tile and cut into one contiguous share per CTA (two CTAs per SM while the row tile is at most
+// tile (the row tiles of one feature tile next to each other, so that their common weight tiles are
+// streamed close together in time) and cut into one contiguous share per CTA (two CTAs per SM while the row tile is at most
 // 128 wide), so every SM streams the same number of weight bytes through long-lived rings whatever
 // n_out is.  A share is a list of segments (tile, k-block range):
 //   warp 0 / lane 0   TMA producer: fills a ring of STAGES {A,B} stages, mbarrier complete_tx
@@ -213,7 +214,7 @@ template <int BN> struct TcCfg {
 
 struct TcParams {
     int kb;                    // k-blocks per tile
-    int n_tiles_m;
+    int n_tiles_n;             // row tiles; tile number = feature tile * n_tiles_n + row tile
     long long units;           // n_tiles_m * n_tiles_n * kb
     int per;                   // units per CTA
     int max_seg;               // scratch slots per CTA
@@ -260,13 +261,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], C::STAGE_BYTES);
-                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM, &full[i]);
+                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM, &full[i]);
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
-                tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[i]);
+                tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[i]);
             }
             int issued = pre;
             for (int i = pre; i < n_units; i++) {
@@ -276,8 +277,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[s], C::STAGE_BYTES);
                 uint8_t* a = smem + s * C::STAGE_BYTES;
-                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM, &full[s]);
-                tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[s]);
+                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM, &full[s]);
+                tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[s]);
                 issued = i + 1;
             }
             if (*abort_flag) {
@@ -410,9 +411,9 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
     const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms);
     if (pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
-    p.kb = pl.kb; p.n_tiles_m = pl.n_tiles_m; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
+    p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
     p.scratch = scratch; p.status = status;
-    out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_m = pl.n_tiles_m; out->bn = pl.bn;
+    out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_n = pl.n_tiles_n; out->bn = pl.bn;
     out->max_seg = pl.max_seg;
     switch (pl.bn_idx) {
         case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);

@@ -335,7 +335,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     const rd_config& c = m->cfg;
     const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
     s->n_slots = sc.batch * sc.max_window;
-    s->R = std::max(s->n_slots, 128);
+    s->R = std::max(s->n_slots, 512);   // prefill chunk: rows that share one pass over the weights
     s->R = (s->R + 15) / 16 * 16;
     s->tok_stride = sc.max_context + 1;
     s->seq_stride = (size_t)sc.max_context * h;

@@ -10,11 +10,12 @@
 
 namespace rd {
 
-// Units (tile, k-block) are numbered tile by tile, kb per tile; CTA g owns units [g*per, (g+1)*per).
+// Tile number = (feature tile) * n_tiles_n + (row tile).  Units (tile, k-block) are numbered tile by
+// tile, kb per tile; CTA g owns units [g*per, (g+1)*per).
 // The j-th tile CTA g touches went to slot g*max_seg + j, laid out [bn rows][128 features].
 struct PartialSums {
     const float* scratch;
-    int kb, per, n_tiles_m, bn, max_seg;
+    int kb, per, n_tiles_n, bn, max_seg;
 };
 
 struct RowSource {
@@ -28,7 +29,7 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     if (s.plain) return *reinterpret_cast<const float4*>(s.plain + (size_t)r * s.ld + m);
     const PartialSums& d = s.part;
     // (unit numbers stay far below 2^31: 32-bit arithmetic)
-    const unsigned tile = (unsigned)(r / d.bn) * d.n_tiles_m + (m >> 7);
+    const unsigned tile = (unsigned)(m >> 7) * d.n_tiles_n + (unsigned)(r / d.bn);
     const unsigned t_lo = tile * (unsigned)d.kb;
     const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
     const size_t in_slot = (size_t)(r % d.bn) * 128 + (m & 127);
