@@ -201,15 +201,24 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     extern __shared__ __align__(16) float xpart[];
     __shared__ float sm[32];
     __shared__ float ss_all[NORM_CLUSTER];                       // every block's sum, pushed by its owner
-    pdl_enter();
+    // the gains are weights: they are fetched before the wait for the predecessor
+    pdl_trigger();
+    const int chunk = ((hidden / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
+    const int m0 = blockIdx.x * chunk, m1 = min(hidden, m0 + chunk);
+    constexpr int GMAX = 4;                                      // gains kept in registers per thread
+    float gr[GMAX];
+#pragma unroll
+    for (int i = 0; i < GMAX; i++) {
+        const int j = m0 + threadIdx.x + i * blockDim.x;
+        gr[i] = j < m1 ? g[j] : 0.f;
+    }
+    pdl_wait();
     cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
     const int r = blockIdx.y;
     if (row_pos && row_pos[r] < 0) return;                       // the whole cluster leaves
     // first cluster barrier, split: arrive now, wait before the first access to another block's
     // shared memory (which is only legal once that block runs)
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    const int chunk = ((hidden / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
-    const int m0 = blockIdx.x * chunk, m1 = min(hidden, m0 + chunk);
     float ss = 0.f;
     for (int m = m0 + threadIdx.x * 4; m < m1; m += blockDim.x * 4) {
         float4 v = row_source_load4(src, r, m);
@@ -233,7 +242,12 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     float tot = 0.f;
     for (int k = 0; k < NORM_CLUSTER; k++) tot += ss_all[k];
     const float inv = 1.0f / sqrtf(tot / (float)hidden + eps);
-    for (int j = m0 + threadIdx.x; j < m1; j += blockDim.x)
+#pragma unroll
+    for (int i = 0; i < GMAX; i++) {
+        const int j = m0 + threadIdx.x + i * blockDim.x;
+        if (j < m1) out[(size_t)r * ldo + j] = from_f<TO>(gr[i] * (xpart[j - m0] * inv));
+    }
+    for (int j = m0 + threadIdx.x + GMAX * blockDim.x; j < m1; j += blockDim.x)
         out[(size_t)r * ldo + j] = from_f<TO>(g[j] * (xpart[j - m0] * inv));
 }
 
@@ -348,17 +362,18 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
                                T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride, size_t head_stride) {
     pdl_enter();
     const int r = blockIdx.x;
-    const int p = row_pos[r];
-    if (p < 0) return;
     const int half = head_dim / 2;
-    // cache layout [sequence][head][position][head_dim]: a head's keys are one contiguous stream
-    T* kseq = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
-    T* vseq = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
     T* qdst = q_t + (size_t)r * hidden;
     // four features = two rotary pairs per thread and turn
     for (int m = (blockIdx.y * blockDim.x + threadIdx.x) * 4; m < hidden; m += gridDim.y * blockDim.x * 4) {
+        // the sums are requested first; the row's position (and with it the rotary angles) meanwhile
         const float4 q = row_source_load4(src, r, m), k = row_source_load4(src, r, hidden + m),
                      v = row_source_load4(src, r, 2 * hidden + m);
+        const int p = row_pos[r];
+        if (p < 0) return;
+        // cache layout [sequence][head][position][head_dim]: a head's keys are one contiguous stream
+        T* kseq = Kc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
+        T* vseq = Vc + (size_t)row_seq[r] * seq_stride + (size_t)p * head_dim;
         const int i0 = ((m % head_dim) >> 1), i1 = (((m + 2) % head_dim) >> 1);
         const float c0 = cos_t[(size_t)p * half + i0], s0 = sin_t[(size_t)p * half + i0];
         const float c1 = cos_t[(size_t)p * half + i1], s1 = sin_t[(size_t)p * half + i1];
@@ -455,8 +470,8 @@ __global__ void swiglu_kernel(const RowSource src, int inner, T* __restrict__ ac
     const size_t quads = (size_t)inner / 4;
     if (i >= (size_t)n_rows * quads) return;
     const int r = (int)(i / quads), j = (int)(i % quads) * 4;
-    if (row_pos[r] < 0) return;
     const float4 g = row_source_load4(src, r, j), u = row_source_load4(src, r, inner + j);
+    if (row_pos[r] < 0) return;
     const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int k = 0; k < 4; k++) act[(size_t)r * lda + j + k] = from_f<T>((gv[k] / (1.0f + expf(-gv[k]))) * uv[k]);
