@@ -120,3 +120,35 @@ def test_gpu_run_to_run_bit_identical():
                      sess.debug_read(rd.RD_DBG_LOGITS, 0).copy()))
     for a, b in zip(outs[0], outs[1]):
         assert np.array_equal(a, b)
+
+
+def test_twin_window_64_rows():
+    """A 64-row wavefront: the 64-row GEMM tile and the four-query-block attention path in decode.
+    A row stays in flight for 64 recurrences here; with the plain random init the recurrence is not
+    contractive and bf16 rounding differences between the two sides grow with every pass, so the
+    latent's share of the adapter is scaled down (contractive recurrence, as for the convergence pin)."""
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 64, 70, max_ctx=256, adapter_s_scale=0.25)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [50], 2, 70)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    widest = 0
+    for _ in range(80):                       # ramp to the full window and a few steps beyond
+        if ls.all_done():
+            break
+        widest = max(widest, len(seqs[0].window))
+        ls.df(64, 1, 0.0)
+    assert widest == 64
+    assert _ties_ok(ls)
+
+
+def test_twin_batch_16_window_16_is_256_rows():
+    """The batched-serving row count: 16 sequences x 16 in-flight rows = the 256-row GEMM tile, ragged
+    prompts, temperature sampling, adaptive exit."""
+    lens = rd_inputs.make_prompt_lengths(16, 2, 40, seed=9)
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 16, 20, batch=16, temperature=1.0, cap=8, max_ctx=128)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 2, 20)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    for _ in range(24):
+        if ls.all_done():
+            break
+        ls.df(16, 1, 1e-3)
+    assert _ties_ok(ls)
