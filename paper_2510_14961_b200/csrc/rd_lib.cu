@@ -233,6 +233,9 @@ struct rd_session {
     int *step_first = nullptr, *step_n = nullptr, *draft = nullptr;
     unsigned long long* counters = nullptr;
     int* status = nullptr;   // device word: non-zero when a bounded wait ran out
+    size_t poll_ints = 0;    // status[4], n_committed[B], done[B] are one device block ...
+    int* mirror = nullptr;   // ... mirrored in pinned host memory by one copy
+    uint64_t enqueue_epoch = 1, mirror_epoch = 0;   // mirror is current while the two are equal
     float *x = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
     float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
     float* tc_scratch = nullptr;   // partial sums of tiles whose K range is shared between CTAs
@@ -260,6 +263,7 @@ struct rd_session {
     std::vector<cudaEvent_t> event_pool;
     uint64_t ctx_total = 0;   // host-side upper bound of sum over sequences of context length
     ~rd_session() {
+        if (mirror) cudaFreeHost(mirror);
         for (Bracket& b : brackets) { cudaEventDestroy(b.a); cudaEventDestroy(b.b); }
         for (cudaEvent_t e : event_pool) cudaEventDestroy(e);
     }
@@ -345,9 +349,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     do {
         if ((rc = s->mem.get(&s->tokens, B * s->tok_stride * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->n_prompt, B * sizeof(int)))) break;
-        if ((rc = s->mem.get(&s->n_committed, B * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->win_len, B * sizeof(int)))) break;
-        if ((rc = s->mem.get(&s->done, B * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->step_first, B * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->step_n, B * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->row_steps, R * sizeof(int)))) break;
@@ -356,7 +358,16 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if ((rc = s->mem.get(&s->row_seq, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->draft, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->counters, 8 * sizeof(unsigned long long)))) break;
-        if ((rc = s->mem.get(&s->status, 4 * sizeof(int)))) break;
+        // what the host polls sits in one block (status word, |y_frozen| and done flag per sequence)
+        // so that one copy into a pinned mirror brings all of it
+        s->poll_ints = 4 + 2 * B;
+        if ((rc = s->mem.get(&s->status, s->poll_ints * sizeof(int)))) break;
+        s->n_committed = s->status + 4;
+        s->done = s->n_committed + B;
+        {
+            cudaError_t eh = cudaHostAlloc((void**)&s->mirror, s->poll_ints * sizeof(int), cudaHostAllocDefault);
+            if (eh != cudaSuccess) { rc = cuda_fail(eh, "cudaHostAlloc", __LINE__); break; }
+        }
         if ((rc = s->mem.get(&s->x, R * h * sizeof(float)))) break;
         s->acc_elems = std::max(R * std::max<size_t>(std::max<size_t>(3 * h, 2 * I), h), (size_t)s->n_slots * V);
         if ((rc = s->mem.get(&s->acc, s->acc_elems * sizeof(float)))) break;
@@ -779,6 +790,7 @@ extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int
         if (prompt[i] < 0 || prompt[i] >= s->m->cfg.vocab) return RD_E_INVALID_ARG;
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::prefill(s, seq, prompt, n_prompt, r)
                                               : Eng<float>::prefill(s, seq, prompt, n_prompt, r);
+    s->enqueue_epoch++;
     if (rc == RD_OK) {
         s->prefilled[seq] = 1; s->wave_open[seq] = 0;
         s->host_prompt_len[seq] = n_prompt; s->host_steps[seq] = 0;
@@ -792,6 +804,7 @@ extern "C" int rd_ar_step(rd_session* s, int32_t r) {
     for (int b = 0; b < s->sc.batch; b++)
         if (s->prefilled[b] && s->wave_open[b]) return RD_E_STATE;
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, 1, r, 0.f, false) : Eng<float>::decode_step(s, 1, r, 0.f, false);
+    s->enqueue_epoch++;
     if (rc == RD_OK) s->stats.ar_steps++;
     return rc;
 }
@@ -802,6 +815,7 @@ extern "C" int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, fl
     if (!any_prefilled(s)) return RD_E_STATE;
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, window, inner_iters, exit_threshold, true)
                                               : Eng<float>::decode_step(s, window, inner_iters, exit_threshold, true);
+    s->enqueue_epoch++;
     if (rc == RD_OK) {
         s->stats.df_steps++;
         if (window > 1)
@@ -812,20 +826,20 @@ extern "C" int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, fl
 
 extern "C" int rd_sync(rd_session* s) {
     if (!s) return RD_E_INVALID_ARG;
-    CU(cudaStreamSynchronize(s->stream));
-    int st[4] = {0, 0, 0, 0};
-    CU(cudaMemcpy(st, s->status, sizeof st, cudaMemcpyDeviceToHost));
-    return st[0] ? RD_E_TIMEOUT : RD_OK;
+    if (s->mirror_epoch != s->enqueue_epoch) {
+        // one copy behind everything enqueued so far, then one wait
+        CU(cudaMemcpyAsync(s->mirror, s->status, s->poll_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+        CU(cudaStreamSynchronize(s->stream));
+        s->mirror_epoch = s->enqueue_epoch;
+    }
+    return s->mirror[0] ? RD_E_TIMEOUT : RD_OK;
 }
 
 extern "C" int rd_committed(rd_session* s, int32_t seq, int32_t* n_tokens, int32_t* done) {
     if (!s || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
     RD_TRY(rd_sync(s));
-    int n = 0, d = 0;
-    CU(cudaMemcpy(&n, s->n_committed + seq, sizeof(int), cudaMemcpyDeviceToHost));
-    CU(cudaMemcpy(&d, s->done + seq, sizeof(int), cudaMemcpyDeviceToHost));
-    if (n_tokens) *n_tokens = n;
-    if (done) *done = s->prefilled[seq] ? d : 0;
+    if (n_tokens) *n_tokens = s->mirror[4 + seq];
+    if (done) *done = s->prefilled[seq] ? s->mirror[4 + s->sc.batch + seq] : 0;
     return RD_OK;
 }
 
