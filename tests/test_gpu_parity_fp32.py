@@ -141,3 +141,30 @@ def test_argument_and_state_errors():
         sess.df_step(2, 1, 0.0)
     n, done = sess.committed(0)
     assert done and n == 3 + 4
+
+
+def test_slot_reuse_while_another_sequence_is_in_flight():
+    """Continuous batching in its minimal form: a finished sequence's slot is prefilled again with a
+    new prompt while the other sequence of the batch is in the middle of its wavefront; both go on in
+    lock step with the oracle (sequences are independent)."""
+    W = 3
+    model, gm, sess, sm = _setup(SMALL, 0, 6, W, batch=2, gain_jitter=0.1)
+    seqs = _prefill_both(sm, sess, SMALL, [7, 12], 2, 6)
+    ls = LockStep(sm, sess, seqs, TOL)
+    while not ls.all_done():                        # first generation of both sequences
+        ls.df(W, 1, 0.0)
+    # sequence 1 starts a new request and gets two steps ahead ...
+    prompt1 = rd_inputs.make_prompt(9, SMALL["vocab"], seed=77)
+    seqs[1] = sm.prefill(1, prompt1, 2, 6)
+    sess.prefill(1, prompt1, 2)
+    ls.df(W, 1, 0.0)
+    ls.df(W, 1, 0.0)
+    assert len(seqs[1].window) > 1                  # sequence 1 has an open wavefront
+    # ... then slot 0 is reused for another request while slot 1 is in flight
+    prompt0 = rd_inputs.make_prompt(5, SMALL["vocab"], seed=78)
+    seqs[0] = sm.prefill(0, prompt0, 3, 6)
+    sess.prefill(0, prompt0, 3)
+    while not ls.all_done():
+        ls.df(W, 1, 0.0)
+    ls.final_tokens_equal()
+    assert ls.near_ties == 0
