@@ -53,6 +53,13 @@ WORKLOADS = {
     "3p5b_layers111_v8192_p512_g64_W32": dict(shape=dict(rd_inputs.SHAPE_3P5B, n_prelude=1, n_core=1, n_coda=1, vocab=8192),
                                               bf16=True, batch=1, prompt=512, gen=64, window=32, inner=1, eps=0.0,
                                               ar_r=4, prefill_r=2, temperature=0.0),
+    # small cases of the two batched configurations (same kernel shapes, 1/1/1 layers), for ncu captures
+    "3p5b_layers111_v8192_b16_p256_g64_W16": dict(shape=dict(rd_inputs.SHAPE_3P5B, n_prelude=1, n_core=1, n_coda=1, vocab=8192),
+                                                  bf16=True, batch=16, prompt=256, gen=64, window=16, inner=1, eps=0.0,
+                                                  ar_r=4, prefill_r=1, temperature=0.0),
+    "3p5b_layers111_v8192_b4_p8192_g64_W32": dict(shape=dict(rd_inputs.SHAPE_3P5B, n_prelude=1, n_core=1, n_coda=1, vocab=8192),
+                                                  bf16=True, batch=4, prompt=8192, gen=64, window=32, inner=1, eps=0.0,
+                                                  ar_r=4, prefill_r=1, temperature=0.0),
 }
 DEFAULT_WORKLOAD = "3p5b_b1_p512_g256_W32"
 
