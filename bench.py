@@ -63,9 +63,9 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "3p5b_b1_p512_g256_W32"
 
-# DRAM bytes (read + write) of one average GEMM launch of a step, from the ncu capture summarised in
-# profiles/gemm_tc_kernel_bn32_3p5b_shapes_W32.md (taken on the 1/1/1-layer case with the same GEMM
-# shapes; the head's traffic scaled by vocabulary).  Valid for the kernel as profiled; set to None
+# DRAM bytes (read + write) of one average GEMM launch of a step, from the ncu capture of the 32-row
+# GEMM summarised under profiles/ (taken on the 1/1/1-layer case with the same GEMM shapes; the head's
+# traffic scaled by vocabulary).  Valid for the kernel as profiled; set to None
 # when the GEMM kernel changes until the counters are taken again.
 NCU_GEMM_TRAFFIC_PER_LAUNCH = {"3p5b_b1_p512_g256_W32": 217.7e6}
 
