@@ -83,10 +83,14 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     const int sp = blockIdx.x, n_splits = gridDim.x, hd = blockIdx.y;
     const int r0 = blockIdx.z * rows_per_group;
     const int nq = min(rows_per_group, n_rows - r0);
-    if (tid < ATT_QMAX) pos_s[tid] = tid < nq ? row_pos[r0 + tid] : -1;
+    // positions of the group's rows; kv_len = 1 + the largest of them
+    __shared__ int warp_max[4];
+    const int my_pos = (tid < ATT_QMAX && tid < nq) ? row_pos[r0 + tid] : -1;
+    if (tid < ATT_QMAX) pos_s[tid] = my_pos;
+    const int wmax = __reduce_max_sync(0xffffffffu, my_pos);
+    if (lane == 0) warp_max[warp] = wmax;
     __syncthreads();
-    int kv_len = 0;
-    for (int i = 0; i < ATT_QMAX; i++) kv_len = max(kv_len, pos_s[i] + 1);
+    const int kv_len = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3])) + 1;
     const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
     const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
     const int seq = row_seq[r0];
