@@ -369,7 +369,9 @@ def run_ours(args):
                      "peak_source": peaks["source"]},
         "attention": {"achieved_gbs": attn_gbs, "launches": prof["attn_launches"],
                       "avg_us": 1e3 * prof["attn_ms"] / max(prof["attn_launches"], 1)},
-        "gemm_share_of_step": prof["gemm_ms"] / (prof_steps * ms_per_step) if ms_per_step else None,
+        "kernel_time_shares": {k: prof[k + "_ms"] / max(prof["gemm_ms"] + prof["attn_ms"] + prof["other_ms"], 1e-9)
+                               for k in ("gemm", "attn", "other")},
+        "gemm_share_of_step": prof["gemm_ms"] / max(prof["gemm_ms"] + prof["attn_ms"] + prof["other_ms"], 1e-9),
         "clocks": clk,
         "e2e": {"value": e2e_tok_s, "unit": "tok/s", "h2d_bytes_per_step": 4.0 * sum(lens) / n_steps_e2e,
                 "d2h_bytes_per_step": d2h / n_steps_e2e, "steps": n_steps_e2e, "prefill_s": e2e_prefill_s,

@@ -197,15 +197,17 @@ int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t layer, int32_
 /* rd_stats -- counters since session creation (host pointer out). */
 int rd_stats(rd_session* s, rd_stats_t* out);
 
-/* rd_profile_enable / rd_profile_read -- measurement aid.  While enabled, every GEMM launch and
- * every attention launch is bracketed by a pair of CUDA events recorded on the session's stream;
+/* rd_profile_enable / rd_profile_read -- measurement aid.  While enabled, every GEMM launch, every
+ * attention launch and every other kernel launch is bracketed by a pair of CUDA events recorded on
+ * the session's stream (which also keeps consecutive kernels from overlapping);
  * rd_profile_read synchronises, sums the elapsed times of the pairs recorded since the last read
  * and resets the list.  Bytes are the algorithmic ones: weight bytes of each GEMM (n_out * K *
  * element size), and for attention the K and V rows each (sequence, layer) must read once.
- * At most 16384 pairs are kept between reads; later launches are then not bracketed. */
+ * At most 32768 pairs are kept between reads; later launches are then not bracketed. */
 typedef struct {
     uint64_t gemm_launches;  double gemm_ms;  uint64_t gemm_weight_bytes;
     uint64_t attn_launches;  double attn_ms;  uint64_t attn_kv_bytes;
+    uint64_t other_launches; double other_ms;
 } rd_profile_t;
 int rd_profile_enable(rd_session* s, int32_t on);
 int rd_profile_read(rd_session* s, rd_profile_t* out);

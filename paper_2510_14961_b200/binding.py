@@ -39,7 +39,8 @@ class RdStats(C.Structure):
 
 class RdProfile(C.Structure):
     _fields_ = [("gemm_launches", C.c_uint64), ("gemm_ms", C.c_double), ("gemm_weight_bytes", C.c_uint64),
-                ("attn_launches", C.c_uint64), ("attn_ms", C.c_double), ("attn_kv_bytes", C.c_uint64)]
+                ("attn_launches", C.c_uint64), ("attn_ms", C.c_double), ("attn_kv_bytes", C.c_uint64),
+                ("other_launches", C.c_uint64), ("other_ms", C.c_double)]
 
 
 class RdError(RuntimeError):

@@ -259,6 +259,7 @@ struct rd_session {
     // measurement aid: event pairs around GEMM (kind 0) and attention (kind 1) launches
     struct Bracket { cudaEvent_t a, b; int kind; uint64_t bytes; };
     bool profiling = false;
+    bool bracket_is_open = false;
     std::vector<Bracket> brackets;
     std::vector<cudaEvent_t> event_pool;
     uint64_t ctx_total = 0;   // host-side upper bound of sum over sequences of context length
@@ -271,7 +272,7 @@ struct rd_session {
 
 // RAII-free helpers: open a bracket before a launch, close it after.
 static int bracket_open(rd_session* s, int kind, uint64_t bytes) {
-    if (!s->profiling || s->brackets.size() >= 16384) return -1;
+    if (!s->profiling || s->brackets.size() >= 32768) return -1;
     rd_session::Bracket b;
     b.kind = kind; b.bytes = bytes;
     for (cudaEvent_t* e : {&b.a, &b.b}) {
@@ -280,11 +281,14 @@ static int bracket_open(rd_session* s, int kind, uint64_t bytes) {
     }
     cudaEventRecord(b.a, s->stream);
     s->brackets.push_back(b);
+    s->bracket_is_open = true;
     return (int)s->brackets.size() - 1;
 }
 static void bracket_close(rd_session* s, int idx) {
-    if (idx >= 0) cudaEventRecord(s->brackets[idx].b, s->stream);
+    if (idx >= 0) { cudaEventRecord(s->brackets[idx].b, s->stream); s->bracket_is_open = false; }
 }
+// A launch outside a GEMM or attention bracket gets a bracket of its own (kind 2).
+static int bracket_other(rd_session* s) { return s->bracket_is_open ? -1 : bracket_open(s, 2, 0); }
 
 // The GEMM kernels need the largest shared-memory carve-out an SM offers.  Every other kernel of a
 // step asks for the same carve-out, so that an SM never has to drain and switch its L1 / shared
@@ -461,14 +465,18 @@ extern "C" int rd_set_launch_chaining(rd_session* s, int32_t on) {
 // Every kernel of a step is a link of one programmatic-dependent-launch chain (rd_common.cuh).
 #define LAUNCH_CLUSTER(s, kern, grid, block, smem, cluster_x, ...)                                 \
     do {                                                                                          \
+        const int br_ = bracket_other(s);                                                         \
         cudaError_t e_ = launch_chained_cluster(kern, dim3 grid, dim3(block), smem, (s)->stream, (s)->chained, cluster_x, __VA_ARGS__); \
         if (e_ != cudaSuccess) return cuda_fail(e_, #kern, __LINE__);                             \
+        bracket_close(s, br_);                                                                    \
         (s)->stats.kernel_launches++;                                                             \
     } while (0)
 #define LAUNCH(s, kern, grid, block, smem, ...)                                                   \
     do {                                                                                          \
+        const int br_ = bracket_other(s);                                                         \
         cudaError_t e_ = launch_chained(kern, dim3(grid), dim3(block), smem, (s)->stream, (s)->chained, __VA_ARGS__); \
         if (e_ != cudaSuccess) return cuda_fail(e_, #kern, __LINE__);                             \
+        bracket_close(s, br_);                                                                    \
         (s)->stats.kernel_launches++;                                                             \
     } while (0)
 
@@ -1014,7 +1022,8 @@ extern "C" int rd_profile_read(rd_session* s, rd_profile_t* out) {
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, b.a, b.b) == cudaSuccess) {
             if (b.kind == 0) { out->gemm_launches++; out->gemm_ms += ms; out->gemm_weight_bytes += b.bytes; }
-            else { out->attn_launches++; out->attn_ms += ms; out->attn_kv_bytes += b.bytes; }
+            else if (b.kind == 1) { out->attn_launches++; out->attn_ms += ms; out->attn_kv_bytes += b.bytes; }
+            else { out->other_launches++; out->other_ms += ms; }
         }
         s->event_pool.push_back(b.a);
         s->event_pool.push_back(b.b);
