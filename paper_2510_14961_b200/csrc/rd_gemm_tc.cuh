@@ -52,7 +52,8 @@ constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
 struct TcWeight {
-    CUtensorMap map;
+    CUtensorMap map;             // box of 128 output features
+    CUtensorMap map2;            // box of 256 output features (two tiles per unit, see TC_MT)
     bool valid = false;
     int n_out = 0, K = 0;
 };
@@ -95,7 +96,9 @@ static inline int tc_encode(CUtensorMap* map, const void* ptr, uint64_t rows, ui
 }
 static inline int tc_make_weight(TcWeight* w, const void* ptr, int n_out, int K) {
     w->valid = false;
-    const int rc = tc_encode(&w->map, ptr, (uint64_t)n_out, (uint64_t)K, TC_BM);
+    int rc = tc_encode(&w->map, ptr, (uint64_t)n_out, (uint64_t)K, TC_BM);
+    if (rc) return rc;
+    rc = tc_encode(&w->map2, ptr, (uint64_t)n_out, (uint64_t)K, 2 * TC_BM);
     if (rc) return rc;
     w->n_out = n_out; w->K = K; w->valid = true;
     return RD_OK;
@@ -197,8 +200,14 @@ __host__ __device__ constexpr uint32_t umma_idesc(int bn) {
 #endif
 constexpr int TC_CTAS_PER_SM = 2;   // while BN <= RD_TC_2CTA_MAX_BN
 
+// Feature tiles per unit.  At 256 rows a stage would otherwise move 32 KB of activations from L2 for
+// 16 KB of weights and the SM's L2 port (about 120 GB/s) becomes the limit; two feature tiles share
+// one activation tile there (two accumulators of 256 columns = all of TMEM, no double buffering).
+template <int BN> struct TcTiles { static constexpr int MT = BN == 256 ? 2 : 1; };
+
 template <int BN> struct TcCfg {
-    static constexpr int A_BYTES = TC_BM * TC_BK * 2;                 // 16 KB
+    static constexpr int MT = TcTiles<BN>::MT;
+    static constexpr int A_BYTES = MT * TC_BM * TC_BK * 2;            // 16 KB per feature tile
     static constexpr int B_BYTES = BN * TC_BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     // Two CTAs per SM with about 100 KB of ring each (measured: two independent producer / MMA
@@ -208,17 +217,18 @@ template <int BN> struct TcCfg {
     static constexpr int RING_KB = BN <= RD_TC_2CTA_MAX_BN ? RD_TC_RING_KB : 200;
     static constexpr int STAGES = (RING_KB * 1024) / STAGE_BYTES > 12 ? 12 : (RING_KB * 1024) / STAGE_BYTES;
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
-    static constexpr int ACC_COLS = BN < 32 ? 32 : BN;                // columns of one accumulator buffer
-    static constexpr int TMEM_COLS = 2 * ACC_COLS;                    // power of two, 64..512
+    static constexpr int ACC_COLS = BN < 32 ? 32 : BN;                // columns of one accumulator
+    static constexpr int NBUF = MT == 1 ? 2 : 1;                      // accumulator sets (a set = MT accumulators)
+    static constexpr int TMEM_COLS = NBUF * MT * ACC_COLS;            // power of two, 64..512
 };
 
 struct TcParams {
     int kb;                    // k-blocks per tile
-    int n_tiles_n;             // row tiles; tile number = feature tile * n_tiles_n + row tile
-    long long units;           // n_tiles_m * n_tiles_n * kb
+    int n_tiles_n;             // row tiles; tile number = (feature tile / MT) * n_tiles_n + row tile
+    long long units;           // tiles * kb
     int per;                   // units per CTA
     int max_seg;               // scratch slots per CTA
-    float* scratch;            // [gridDim.x * max_seg][BN][128] partial sums
+    float* scratch;            // [gridDim.x * max_seg][MT][BN][128] partial sums
     int* status;
 };
 
@@ -261,7 +271,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], C::STAGE_BYTES);
-                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM, &full[i]);
+                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM * C::MT, &full[i]);
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
@@ -277,7 +287,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[s], C::STAGE_BYTES);
                 uint8_t* a = smem + s * C::STAGE_BYTES;
-                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM, &full[s]);
+                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM * C::MT, &full[s]);
                 tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[s]);
                 issued = i + 1;
             }
@@ -305,10 +315,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     const long long u = u0 + i;
                     const int ka = (int)(u % p.kb);
                     const int len = min(p.kb - ka, n_units - i);
-                    const int buf = seg & 1;
-                    if (seg >= 2 && !mbar_wait(&acc_empty[buf], ((seg >> 1) - 1) & 1)) { ok = false; break; }
+                    const int buf = seg % C::NBUF, use = seg / C::NBUF;
+                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t d = tmem_base + (uint32_t)(buf * C::ACC_COLS);
+                    const uint32_t d = tmem_base + (uint32_t)(buf * C::MT * C::ACC_COLS);
                     for (int j = 0; j < len; j++, i++) {
                         const int s = i % C::STAGES;
                         if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1)) { ok = false; break; }
@@ -317,7 +327,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
 #pragma unroll
                         for (int k = 0; k < TC_BK / 16; k++)
-                            umma_bf16(d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (j | k) ? 1u : 0u);
+#pragma unroll
+                            for (int mt = 0; mt < C::MT; mt++)   // the mt-th feature tile starts 16 KB further on
+                                umma_bf16(d + (uint32_t)(mt * C::ACC_COLS), adesc + (uint64_t)(mt * 1024 + k * 2),
+                                          bdesc + (uint64_t)(k * 2), idesc, (j | k) ? 1u : 0u);
                         umma_commit(&empty[s]);          // stage reusable once these MMAs have read it
                     }
                     if (!ok) break;
@@ -335,16 +348,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const long long u = u0 + i;
                 const int ka = (int)(u % p.kb);
                 const int len = min(p.kb - ka, n_units - i);
-                const int buf = seg & 1;
-                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg >> 1) & 1)) { ok = false; break; }
+                const int buf = seg % C::NBUF;
+                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_COLS);
+                const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::MT * C::ACC_COLS);
                 // the share's seg-th segment (= seg-th tile it touches) -> slot blockIdx.x * max_seg + seg
-                float* slot = p.scratch + ((size_t)blockIdx.x * p.max_seg + seg) * (size_t)(BN * TC_BM) + quad * 32 + lane;
+                float* slot = p.scratch + ((size_t)blockIdx.x * p.max_seg + seg) * (size_t)(C::MT * BN * TC_BM) + quad * 32 + lane;
 #pragma unroll 1
-                for (int c = 0; c < BN; c += 16) {
+                for (int c = 0; c < C::MT * BN; c += 16) {      // column c = (feature tile in the unit) * BN + row
                     uint32_t raw[16];
-                    tmem_ld16(t + (uint32_t)c, raw);
+                    tmem_ld16(t + (uint32_t)((c / BN) * C::ACC_COLS + c % BN), raw);
 #pragma unroll
                     for (int j = 0; j < 16; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
                 }
@@ -369,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 static inline int tc_pick_bn(int n_rows) { return n_rows <= 16 ? 0 : n_rows <= 32 ? 1 : n_rows <= 64 ? 2 : n_rows <= 128 ? 3 : 4; }
 
 struct TcPlan {
-    int bn_idx, bn, kb, n_tiles_m, n_tiles_n, per, grid, max_seg;
+    int bn_idx, bn, mt, kb, n_tiles_m, n_tiles_n, per, grid, max_seg;
     long long units;
     size_t scratch_elems;
 };
@@ -380,14 +393,15 @@ static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms) {
     pl.bn = 16 << pl.bn_idx;
     if (pl.bn <= RD_TC_2CTA_MAX_BN) n_sms *= TC_CTAS_PER_SM;
     pl.kb = (K + TC_BK - 1) / TC_BK;
-    pl.n_tiles_m = (n_out + TC_BM - 1) / TC_BM;
+    pl.mt = pl.bn == 256 ? 2 : 1;                       // = TcTiles<bn>::MT
+    pl.n_tiles_m = (n_out + pl.mt * TC_BM - 1) / (pl.mt * TC_BM);   // units cover mt feature tiles
     pl.n_tiles_n = (n_rows + pl.bn - 1) / pl.bn;
     pl.units = (long long)pl.n_tiles_m * pl.n_tiles_n * pl.kb;
     const long long g = std::min<long long>(n_sms, pl.units);
     pl.per = (int)((pl.units + g - 1) / g);
     pl.grid = (int)((pl.units + pl.per - 1) / pl.per);
     pl.max_seg = (pl.per + pl.kb - 1) / pl.kb + 1;      // tiles a run of `per` units can touch
-    pl.scratch_elems = (size_t)pl.grid * pl.max_seg * pl.bn * TC_BM;
+    pl.scratch_elems = (size_t)pl.grid * pl.max_seg * pl.mt * pl.bn * TC_BM;
     return pl;
 }
 
@@ -414,13 +428,13 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
     p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
     p.scratch = scratch; p.status = status;
     out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_n = pl.n_tiles_n; out->bn = pl.bn;
-    out->max_seg = pl.max_seg;
+    out->max_seg = pl.max_seg; out->mt_shift = pl.mt == 2 ? 1 : 0;
     switch (pl.bn_idx) {
         case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);
         case 1: return tc_launch<32>(st, tw.map, ta.map[1], p, pl.grid, chained);
         case 2: return tc_launch<64>(st, tw.map, ta.map[2], p, pl.grid, chained);
         case 3: return tc_launch<128>(st, tw.map, ta.map[3], p, pl.grid, chained);
-        default: return tc_launch<256>(st, tw.map, ta.map[4], p, pl.grid, chained);
+        default: return tc_launch<256>(st, tw.map2, ta.map[4], p, pl.grid, chained);
     }
 }
 

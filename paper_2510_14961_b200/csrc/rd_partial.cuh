@@ -10,12 +10,13 @@
 
 namespace rd {
 
-// Tile number = (feature tile) * n_tiles_n + (row tile).  Units (tile, k-block) are numbered tile by
+// Tile number = (feature tile >> mt_shift) * n_tiles_n + (row tile).  Units (tile, k-block) are numbered tile by
 // tile, kb per tile; CTA g owns units [g*per, (g+1)*per).
-// The j-th tile CTA g touches went to slot g*max_seg + j, laid out [bn rows][128 features].
+// The j-th tile CTA g touches went to slot g*max_seg + j, laid out [feature tile][bn rows][128 features].
 struct PartialSums {
     const float* scratch;
     int kb, per, n_tiles_n, bn, max_seg;
+    int mt_shift;         // a tile covers 1 << mt_shift feature tiles of 128 (slot: [feature tile][bn rows][128])
 };
 
 struct RowSource {
@@ -29,12 +30,13 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     if (s.plain) return *reinterpret_cast<const float4*>(s.plain + (size_t)r * s.ld + m);
     const PartialSums& d = s.part;
     // (unit numbers stay far below 2^31: 32-bit arithmetic)
-    const unsigned tile = (unsigned)(m >> 7) * d.n_tiles_n + (unsigned)(r / d.bn);
+    const unsigned ft = (unsigned)(m >> 7);
+    const unsigned tile = (ft >> d.mt_shift) * d.n_tiles_n + (unsigned)(r / d.bn);
     const unsigned t_lo = tile * (unsigned)d.kb;
     const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
-    const size_t in_slot = (size_t)(r % d.bn) * 128 + (m & 127);
+    const size_t in_slot = ((size_t)(ft & ((1u << d.mt_shift) - 1)) * d.bn + (size_t)(r % d.bn)) * 128 + (m & 127);
     const float* base = d.scratch + in_slot;
-    const size_t slot_elems = (size_t)d.bn * 128;
+    const size_t slot_elems = ((size_t)d.bn * 128) << d.mt_shift;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     // up to eight slots are requested together (one round trip to L2), then added in ascending k order
     for (int gb = g_lo; gb <= g_hi; gb += 8) {
