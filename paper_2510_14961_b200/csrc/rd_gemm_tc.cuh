@@ -30,6 +30,10 @@
 // do not depend on earlier kernels), and only then waits for the predecessor before touching
 // activations or the scratch buffer.
 //
+// Tiles of 256 rows run on CTA pairs (gemm_tc_pair_kernel, tcgen05 cta_group::2): the two CTAs of a
+// cluster each stage one 128-feature weight tile and half of the rows, and one MMA of M = 256 spans
+// both SMs.  Same units, slots and consumers.
+//
 // Every wait on an mbarrier is bounded; on time-out the kernel raises a status word, drains the
 // copies it issued, frees its TMEM and returns.
 #pragma once
@@ -166,6 +170,53 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// ---- CTA-pair (cta_group::2) forms: two CTAs of a cluster, one on each SM of a pair, run one MMA
+// of M = 256; the even-ranked CTA (the leader) issues it and owns the barriers the loads signal ----
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(const void* p, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on a barrier of the pair's leader
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
+// issued by the same warp of both CTAs of the pair, with the same shared-memory offset for the result
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives, once the pair's MMAs issued so far have completed, on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(both) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
@@ -173,6 +224,19 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// 32 columns of this warp's 32 lanes in one instruction (fewer load/wait round trips per segment)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -188,8 +252,8 @@ __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t umma_idesc(int bn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t umma_idesc(int bn, int m = TC_BM) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 #ifndef RD_TC_RING_KB
@@ -354,12 +418,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::MT * C::ACC_COLS);
                 // the share's seg-th segment (= seg-th tile it touches) -> slot blockIdx.x * max_seg + seg
                 float* slot = p.scratch + ((size_t)blockIdx.x * p.max_seg + seg) * (size_t)(C::MT * BN * TC_BM) + quad * 32 + lane;
+                if constexpr (BN >= 32) {
 #pragma unroll 1
-                for (int c = 0; c < C::MT * BN; c += 16) {      // column c = (feature tile in the unit) * BN + row
-                    uint32_t raw[16];
-                    tmem_ld16(t + (uint32_t)((c / BN) * C::ACC_COLS + c % BN), raw);
+                    for (int c = 0; c < C::MT * BN; c += 32) {  // column c = (feature tile in the unit) * BN + row
+                        uint32_t raw[32];
+                        tmem_ld32(t + (uint32_t)((c / BN) * C::ACC_COLS + c % BN), raw);
 #pragma unroll
-                    for (int j = 0; j < 16; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
+                        for (int j = 0; j < 32; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
+                    }
+                } else {
+                    uint32_t raw[16];
+                    tmem_ld16(t, raw);
+#pragma unroll
+                    for (int j = 0; j < 16; j++) slot[(size_t)j * TC_BM] = __uint_as_float(raw[j]);
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -379,6 +450,189 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// 256-row tiles on a CTA pair.  Two CTAs of a cluster (one per SM of a pair) share every unit: a unit
+// is (256 output features, 256 rows, one k-block); CTA `rank` loads the rank-th 128-feature weight
+// tile and the rank-th 128 rows of the activation tile, the leader (rank 0) issues one MMA of
+// M = 256, N = 256 per K = 16 slice, and each CTA's TMEM receives its own 128 features x 256 rows.
+// Against one CTA running two M = 128 MMAs over a full 256-row activation tile, each SM stages half
+// the activation bytes per weight byte (32 KB instead of 48 KB of shared-memory writes per k-block and
+// each half of the activation tile is read from shared memory once for both tensor cores), and the ring is 6 deep.
+//   full[s]       leader's, 1 arrival + the bytes of both CTAs' loads (the loads of the other CTA name
+//                 the leader's barrier)
+//   empty[s]      one in each CTA, released by the leader's tcgen05.commit to both
+//   acc_full[b]   one in each CTA, same
+//   acc_empty[b]  leader's, 8 arrivals: the four TMEM-reading warps of both CTAs
+// Slots, segments and the consumer side are those of gemm_tc_kernel<256>, with a pair in place of a CTA.
+// ---------------------------------------------------------------------------------------------
+struct TcPairCfg {
+    static constexpr int BN = 256;                                    // rows of a unit (UMMA N)
+    static constexpr int A_BYTES = TC_BM * TC_BK * 2;                 // this CTA's weight tile, 16 KB
+    static constexpr int B_BYTES = (BN / 2) * TC_BK * 2;              // this CTA's half of the rows, 16 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = 6;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int ACC_COLS = BN;
+    static constexpr int NBUF = 2;
+    static constexpr int TMEM_COLS = NBUF * ACC_COLS;                 // 512: all of TMEM, one CTA per SM
+};
+
+__global__ void __launch_bounds__(TC_THREADS)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const TcParams p) {
+    using C = TcPairCfg;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = (uint64_t*)(smem + C::STAGES * C::STAGE_BYTES);
+    uint64_t* empty = full + C::STAGES;
+    uint64_t* acc_full = empty + C::STAGES;     // [2]
+    uint64_t* acc_empty = acc_full + 2;         // [2]
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();       // 0: leader
+    const int pair = blockIdx.x >> 1;
+    const long long u0 = (long long)pair * p.per;
+    const long long u1 = min(p.units, u0 + p.per);
+    pdl_trigger();
+    if (u0 >= u1) { pdl_wait(); return; }       // no share for this pair (both CTAs leave together)
+    const int n_units = (int)(u1 - u0);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    cluster_sync_all();                         // both CTAs' barriers exist before anything signals them
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer (one in each CTA) ----
+            const int pre = min(n_units, C::STAGES);
+            for (int i = 0; i < pre; i++) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                if (rank == 0) mbar_expect_tx(&full[i], 2 * C::STAGE_BYTES);
+                tma_load_2d_pair(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK,
+                                 ((tile / p.n_tiles_n) * 2 + (int)rank) * TC_BM, map_to_rank(&full[i], 0));
+            }
+            pdl_wait();
+            for (int i = 0; i < pre; i++) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                tma_load_2d_pair(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK,
+                                 (tile % p.n_tiles_n) * C::BN + (int)rank * (C::BN / 2), map_to_rank(&full[i], 0));
+            }
+            int issued = pre;
+            for (int i = pre; i < n_units; i++) {
+                const int s = i % C::STAGES;
+                if (*abort_flag || !mbar_wait(&empty[s], ((i / C::STAGES) - 1) & 1)) { *abort_flag = 1; break; }
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
+                if (rank == 0) mbar_expect_tx(&full[s], 2 * C::STAGE_BYTES);
+                uint8_t* a = smem + s * C::STAGE_BYTES;
+                const uint32_t bar = map_to_rank(&full[s], 0);
+                tma_load_2d_pair(a, &tmap_w, kblk * TC_BK, ((tile / p.n_tiles_n) * 2 + (int)rank) * TC_BM, bar);
+                tma_load_2d_pair(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * C::BN + (int)rank * (C::BN / 2), bar);
+                issued = i + 1;
+            }
+            if (*abort_flag && rank == 0) {
+                // drain: the stages the leader armed count both CTAs' bytes
+                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1);
+            }
+        } else {
+            pdl_wait();
+        }
+    } else {
+        if (warp == 1) tmem_alloc_pair(tmem_slot, C::TMEM_COLS);
+        tc_fence_before();
+        named_bar_sync(1, TC_THREADS - 32);
+        tc_fence_after();
+        const uint32_t tmem_base = *tmem_slot;
+        pdl_wait();
+        if (warp == 1) {
+            if (lane == 0 && rank == 0) {
+                // ---- MMA issuer (leader only) ----
+                constexpr uint32_t idesc = umma_idesc(C::BN, 2 * TC_BM);
+                int i = 0, seg = 0;
+                bool ok = true;
+                while (i < n_units && ok) {
+                    const long long u = u0 + i;
+                    const int ka = (int)(u % p.kb);
+                    const int len = min(p.kb - ka, n_units - i);
+                    const int buf = seg % C::NBUF, use = seg / C::NBUF;
+                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d = tmem_base + (uint32_t)(buf * C::ACC_COLS);
+                    for (int j = 0; j < len; j++, i++) {
+                        const int s = i % C::STAGES;
+                        if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a = smem_u32(smem + s * C::STAGE_BYTES);
+                        const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
+#pragma unroll
+                        for (int k = 0; k < TC_BK / 16; k++)
+                            umma_bf16_pair(d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (j | k) ? 1u : 0u);
+                        umma_commit_pair(&empty[s]);         // both CTAs' stage s reusable once these MMAs have read it
+                    }
+                    if (!ok) break;
+                    umma_commit_pair(&acc_full[buf]);        // this segment's sums are complete in both CTAs
+                    seg++;
+                }
+                if (!ok) *abort_flag = 1;
+            }
+        } else {
+            // ---- warps 2..5 of both CTAs move their 128 features of a finished segment to its slot ----
+            const int quad = warp & 3;
+            const uint32_t leader_empty0 = map_to_rank(&acc_empty[0], 0), leader_empty1 = map_to_rank(&acc_empty[1], 0);
+            int i = 0, seg = 0;
+            bool ok = true;
+            while (i < n_units && ok) {
+                const long long u = u0 + i;
+                const int ka = (int)(u % p.kb);
+                const int len = min(p.kb - ka, n_units - i);
+                const int buf = seg % C::NBUF;
+                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_COLS);
+                // slot of the pair's seg-th segment; this CTA's feature tile is the rank-th of the unit's two
+                float* slot = p.scratch + ((size_t)pair * p.max_seg + seg) * (size_t)(2 * C::BN * TC_BM) +
+                              (size_t)rank * (C::BN * TC_BM) + quad * 32 + lane;
+#pragma unroll 1
+                for (int c = 0; c < C::BN; c += 32) {
+                    uint32_t raw[32];
+                    tmem_ld32(t + (uint32_t)c, raw);
+#pragma unroll
+                    for (int j = 0; j < 32; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(buf ? leader_empty1 : leader_empty0);
+                i += len;
+                seg++;
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        atomicExch(p.status, 1);
+        // the other CTA's loads into its own memory are counted on the leader's barriers only:
+        // give copies still in flight time to land before this CTA's memory is released
+        if (rank != 0) for (int i = 0; i < 200; i++) __nanosleep(1000);
+    }
+    __syncthreads();
+    cluster_sync_all();                         // nobody signals or reads a CTA that has left
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(*tmem_slot, C::TMEM_COLS);
+    }
+}
+
 static inline int tc_pick_bn(int n_rows) { return n_rows <= 16 ? 0 : n_rows <= 32 ? 1 : n_rows <= 64 ? 2 : n_rows <= 128 ? 3 : 4; }
 
 struct TcPlan {
@@ -387,11 +641,13 @@ struct TcPlan {
     size_t scratch_elems;
 };
 // Every CTA gets `per` consecutive units (the last ones possibly fewer).
-static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms) {
+// `pair`: 256-row tiles go to CTA pairs (gemm_tc_pair_kernel) instead of single CTAs.
+static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair = true) {
     TcPlan pl;
     pl.bn_idx = tc_pick_bn(n_rows);
     pl.bn = 16 << pl.bn_idx;
     if (pl.bn <= RD_TC_2CTA_MAX_BN) n_sms *= TC_CTAS_PER_SM;
+    else if (pair) n_sms /= 2;                          // a CTA pair per two SMs takes a share
     pl.kb = (K + TC_BK - 1) / TC_BK;
     pl.mt = pl.bn == 256 ? 2 : 1;                       // = TcTiles<bn>::MT
     pl.n_tiles_m = (n_out + pl.mt * TC_BM - 1) / (pl.mt * TC_BM);   // units cover mt feature tiles
@@ -417,12 +673,24 @@ static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& 
                ? RD_OK : RD_E_CUDA;
 }
 
+static int tc_launch_pair(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, int pairs, bool chained) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TcPairCfg::SMEM) != cudaSuccess)
+            return RD_E_CUDA;
+        attr_set = true;
+    }
+    return launch_chained_cluster(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(TC_THREADS), TcPairCfg::SMEM, st, chained, 2, mw, mx, p) ==
+                   cudaSuccess ? RD_OK : RD_E_CUDA;
+}
+
 // Launches the GEMM; *out describes where a consumer finds the sums.  Returns RD_E_INVALID_ARG when
 // the shape is not taken (caller falls back to the SIMT kernels).
 static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
-                          float* scratch, size_t scratch_elems, int n_sms, int* status, bool chained, PartialSums* out) {
+                          float* scratch, size_t scratch_elems, int n_sms, int* status, bool chained, PartialSums* out,
+                          bool pair = true) {
     if (ta.K != K || tw.K != K || tw.n_out != n_out || n_rows < 1 || n_rows > ta.rows) return RD_E_INVALID_ARG;
-    const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms);
+    const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms, pair);
     if (pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
     p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
@@ -434,7 +702,9 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
         case 1: return tc_launch<32>(st, tw.map, ta.map[1], p, pl.grid, chained);
         case 2: return tc_launch<64>(st, tw.map, ta.map[2], p, pl.grid, chained);
         case 3: return tc_launch<128>(st, tw.map, ta.map[3], p, pl.grid, chained);
-        default: return tc_launch<256>(st, tw.map2, ta.map[4], p, pl.grid, chained);
+        default:
+            if (pair) return tc_launch_pair(st, tw.map, ta.map[3], p, pl.grid, chained);
+            return tc_launch<256>(st, tw.map2, ta.map[4], p, pl.grid, chained);
     }
 }
 

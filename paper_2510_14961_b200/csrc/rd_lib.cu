@@ -422,7 +422,9 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
             size_t need = 16;
             for (int nr = 16; ; nr *= 2) {
                 const int rows = std::min<int>(nr, (int)R);
-                for (auto& sh : shapes) need = std::max(need, tc_plan(sh[0], sh[1], rows, m->n_sms).scratch_elems);
+                for (auto& sh : shapes)
+                    for (int pair = 0; pair < 2; pair++)     // either choice of rd_set_gemm_path
+                        need = std::max(need, tc_plan(sh[0], sh[1], rows, m->n_sms, pair != 0).scratch_elems);
                 if (nr >= (int)R) break;
             }
             s->tc_scratch_elems = need;
@@ -447,8 +449,8 @@ extern "C" void rd_session_destroy(rd_session* s) {
     delete s;
 }
 extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
-    if (!s || (path != 0 && path != 1)) return RD_E_INVALID_ARG;
-    if (path == 1 && !(s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
+    if (!s || path < 0 || path > 2) return RD_E_INVALID_ARG;
+    if (path >= 1 && !(s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
     s->gemm_path = path;
     return RD_OK;
 }
@@ -494,7 +496,7 @@ static Pending plain_rows(const float* x, size_t ld) {
 
 template <typename T> struct Eng {
     static bool tc_usable(const rd_session* s, const TcAct* ta, const TcWeight* tw) {
-        return sizeof(T) == 2 && s->gemm_path == 1 && ta && tw && ta->valid && tw->valid;
+        return sizeof(T) == 2 && s->gemm_path >= 1 && ta && tw && ta->valid && tw->valid;
     }
 
     // acc[r, o] = sum_k A[r, k] W[o, k]; *out tells the consumer where the sums are: partial sums of
@@ -505,7 +507,7 @@ template <typename T> struct Eng {
         *out = RowSource{};
         if (tc_usable(s, ta, tw)) {
             const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, n_rows, s->tc_scratch, s->tc_scratch_elems, s->m->n_sms,
-                                   s->status, s->chained, &out->part);
+                                   s->status, s->chained, &out->part, s->gemm_path == 1);
             if (rc == RD_OK) {
                 s->stats.tc_gemm_launches++; s->stats.kernel_launches++;
                 bracket_close(s, br);

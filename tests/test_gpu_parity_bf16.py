@@ -140,11 +140,13 @@ def test_twin_window_64_rows():
     assert _ties_ok(ls)
 
 
-def test_twin_batch_16_window_16_is_256_rows():
-    """The batched-serving row count: 16 sequences x 16 in-flight rows = the 256-row GEMM tile, ragged
-    prompts, temperature sampling, adaptive exit."""
+@pytest.mark.parametrize("path", [1, 2])
+def test_twin_batch_16_window_16_is_256_rows(path):
+    """The batched-serving row count: 16 sequences x 16 in-flight rows = the 256-row GEMM tile (path 1:
+    on CTA pairs, one MMA of 256 features over two SMs; path 2: on single CTAs), ragged prompts,
+    temperature sampling, adaptive exit."""
     lens = rd_inputs.make_prompt_lengths(16, 2, 40, seed=9)
-    model, gm, sess, sm = _setup(rd_inputs.TWIN, 16, 20, batch=16, temperature=1.0, cap=8, max_ctx=128)
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 16, 20, batch=16, temperature=1.0, cap=8, max_ctx=128, gemm_path=path)
     seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 2, 20)
     ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
     for _ in range(24):
@@ -152,3 +154,4 @@ def test_twin_batch_16_window_16_is_256_rows():
             break
         ls.df(16, 1, 1e-3)
     assert _ties_ok(ls)
+    assert sess.stats()["tc_gemm_launches"] > 0      # no silent fall-back to the plain kernels
