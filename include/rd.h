@@ -75,7 +75,7 @@ typedef struct {
     float eta;                 /* Section 3.4: momentum on the input conditioning of rd_df_step,
                                   e = eta e_prev + (1 - eta) P(y_current) from a position's second
                                   step on; 0 <= eta < 1, 0 = off                                  */
-    float beta;                /* Section 3.4 / Algorithm 1 lines 6-7: latent noise in rd_df_step,
+    float beta;                /* Section 3.4 / the stabiliser steps of Algorithm 1: latent noise in rd_df_step,
                                   z <- (1 - b_t) z + b_t z_noise, b_t = beta max(0, 1 - t / T) at a
                                   position's step t; T = window (fixed exit) or
                                   ceil(max_iters_per_pos / inner_iters); 0 <= beta <= 1, 0 = off  */
@@ -116,8 +116,8 @@ void rd_session_destroy(rd_session* s);
 
 /* rd_prefill -- Section 3.3: positions 0..n_prompt-2 of sequence `seq` run P, `r` simultaneous
  * passes of R (pass i of position p attends pass-i K/V of positions <= p) and the coda layers;
- * position n_prompt-1 becomes the first in-flight position with a fresh state (Algorithm 1,
- * lines 1-3).  prompt: host pointer to n_prompt token ids in [0, vocab).  Re-prefilling a
+ * position n_prompt-1 becomes the first in-flight position with a fresh state (the initialisation
+ * steps of Algorithm 1).  prompt: host pointer to n_prompt token ids in [0, vocab).  Re-prefilling a
  * sequence restarts it.  Errors: INVALID_ARG, CAPACITY (n_prompt + max_new_tokens >
  * max_context), OOM, CUDA. */
 int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r);

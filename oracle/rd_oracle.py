@@ -19,7 +19,9 @@ What follows the paper and where:
 * diffusion-forcing sampler, fixed exit -- Algorithm 1; adaptive exit --
   Eq. 3 (delta_i and k*) and Algorithm 2; wavefront limiter -- Section 3.5.
 * stabilisers: momentum on the conditioning and scheduled latent noise --
-  Section 3.4 (both displays), Algorithm 1 lines 6-7.
+  Section 3.4 (both displays) and the two stabiliser steps of Algorithm 1.
+* Sample: greedy, temperature, top-p -- Algorithms 1-2 name it; the Appendix
+  gives the settings of the evaluation (temperature 0.2, top-p 0.95).
 
 The paper does not print the layer internals; the reading used here (pre-norm
 residual layers, RMSNorm, rotary embedding on adjacent pairs, SwiGLU, one
@@ -36,7 +38,9 @@ Pins (tests/test_oracle_*.py): Philox known-answer vectors; layer math against
 an independent per-element loop and against torch's attention on a full causal
 sequence; cache against a no-cache recomputation; causality; AR == DF(W=1,
 r'=r); first-token identity DF(W, r') vs AR(r = W r'); progress and window
-bounds; pass counters of the cost remark; contraction => adaptive DF == AR.
+bounds; pass counters of the cost remark; contraction => adaptive DF == AR;
+top-p against a hand-worked distribution, a search over all subsets, and the
+sampled frequencies.
 Parity unpinned: quality of the sampler's text (needs trained weights).
 """
 from __future__ import annotations
@@ -135,13 +139,34 @@ def gumbel_noise(seed, seq, token_pos, vocab):
     return -np.log(-np.log(u))
 
 
-def sample_token(logits, temperature, seed, seq, token_pos):
+def nucleus(logits, temperature, top_p):
+    """Boolean mask of the tokens top-p sampling keeps (Appendix, sampling settings of the
+    evaluation: temperature 0.2, top-p 0.95): tokens in descending order of probability under
+    softmax(logits / T) up to and including the first at which the cumulative probability reaches
+    top_p; tokens whose logit equals that of the last one kept are kept with it."""
+    l = np.asarray(logits).astype(np.float32).astype(np.float64)
+    if top_p >= 1.0:
+        return np.ones(l.shape[0], dtype=bool)
+    q = np.exp((l - l.max()) / float(temperature))
+    q /= q.sum()
+    order = np.argsort(-l, kind="stable")
+    cum = np.cumsum(q[order])
+    k = int(np.searchsorted(cum, top_p, side="left"))      # first rank whose cumulative mass >= top_p
+    k = min(k, l.shape[0] - 1)
+    return l >= l[order[k]]
+
+
+def sample_token(logits, temperature, seed, seq, token_pos, top_p=1.0):
     """Sample(p) of Algorithms 1-2.  Greedy (temperature 0): arg max, lowest index on ties.
-    Otherwise the Gumbel-max form of sampling from softmax(logits / T), decided in float32."""
+    Otherwise the Gumbel-max form of sampling from softmax(logits / T), decided in float32; with
+    top_p < 1 the arg max runs over the tokens of `nucleus` only, which samples from the
+    distribution renormalised over them."""
     l32 = np.asarray(logits).astype(np.float32)
     if temperature <= 0.0:
         return int(np.argmax(l32))
     score = l32 / np.float32(temperature) + gumbel_noise(seed, seq, token_pos, l32.shape[0])
+    if top_p < 1.0:
+        score = np.where(nucleus(l32, temperature, top_p), score, -np.inf)
     return int(np.argmax(score))
 
 
@@ -317,7 +342,7 @@ class Sequence:
 
 
 class Sampler:
-    def __init__(self, model: RDModel, seed=0, temperature=0.0, max_iters_per_pos=64, eta=0.0, beta=0.0):
+    def __init__(self, model: RDModel, seed=0, temperature=0.0, max_iters_per_pos=64, eta=0.0, beta=0.0, top_p=1.0):
         """eta: momentum on the input conditioning, e = eta e_prev + (1 - eta) P(y_current)
         (Section 3.4, first display); a position's first step has no e_prev and takes P(.) as is.
         beta: latent noise, z' = (1 - beta_t) z + beta_t z_noise (second display), beta_t falling
@@ -329,18 +354,19 @@ class Sampler:
         self.cap = max_iters_per_pos
         self.eta = eta
         self.beta = beta
+        self.top_p = top_p
 
     def _init(self, seq_id, pos):
         c = self.m.cfg
         return init_state(self.seed, seq_id, pos, c.hidden, c.init_sigma, self.m.dtype)
 
     def _sample(self, logits, seq_id, token_pos):
-        return sample_token(logits, self.temperature, self.seed, seq_id, token_pos)
+        return sample_token(logits, self.temperature, self.seed, seq_id, token_pos, self.top_p)
 
     def prefill(self, seq_id, prompt, r, max_new):
         """Section 3.3: the prompt's positions 0..L-2 run P, r simultaneous passes of R and the
         coda layers (to fill its cache).  Position L-1 becomes the first in-flight position with
-        a fresh state (Algorithm 1, lines 1-3)."""
+        a fresh state (the initialisation steps of Algorithm 1)."""
         prompt = np.asarray(prompt, dtype=np.int64)
         L = len(prompt)
         assert L >= 1 and L + max_new <= self.m.max_ctx
