@@ -182,6 +182,10 @@ def run_ours(args):
     wl = dict(WORKLOADS[args.workload])
     if args.prefill_r > 0:
         wl["prefill_r"] = args.prefill_r
+    if args.temperature >= 0.0:
+        wl["temperature"] = args.temperature
+    if args.top_p > 0.0:
+        wl["top_p"] = args.top_p
     if args.window > 0:
         wl["window"] = args.window
     if args.inner > 0:
@@ -208,7 +212,8 @@ def run_ours(args):
 
     def new_session(window, temperature=0.0):
         return rd.Session(model, batch=B, max_context=max_ctx, max_window=window, max_iters_per_pos=64,
-                          max_new_tokens=N, temperature=temperature, seed=1234, stream=stream.cuda_stream)
+                          max_new_tokens=N, temperature=temperature, seed=1234, stream=stream.cuda_stream,
+                          top_p=wl.get("top_p", 0.0))
 
     def prefill(sess):
         for b in range(B):
@@ -351,6 +356,7 @@ def run_ours(args):
         "config": {"workload": args.workload, "batch": B, "prompt": L if len(set(lens)) == 1 else lens, "generate": N, "window": W,
                    "steps_per_generation": steps_per_gen, "tokens_per_step": tokens_all / (world * K) if K else None,
                    "inner_iters": wl["inner"], "exit_threshold": wl["eps"], "ar_r": wl["ar_r"],
+                   "temperature": wl["temperature"], "top_p": wl.get("top_p", 0.0),
                    "l2": "inputs larger than L2 (weights streamed per step: %.2f GB)" % (step_b / 1e9),
                    "multi_gpu": "replicas only (no data-path collective)"},
         "df_tok_s": df_tok_s, "ar_tok_s": ar_tok_s, "df_over_ar": df_tok_s / ar_tok_s if ar_tok_s else None,
@@ -423,7 +429,7 @@ def oracle_steps(workload, n_steps, budget_s=25.0):
     L = 16 if big else wl["prompt"]
     W = wl["window"]
     model = orc.RDModel(cfg, w, dtype=np.float32 if big else np.float64, contract=False, max_ctx=L + wl["gen"] + 8)
-    sm = orc.Sampler(model, seed=1234, temperature=wl["temperature"])
+    sm = orc.Sampler(model, seed=1234, temperature=wl["temperature"], top_p=wl.get("top_p", 0.0) or 1.0)
     prompt = rd_inputs.make_prompt(L, shape["vocab"], seed=17)
     sq = sm.prefill(0, prompt, 1 if big else wl["prefill_r"], wl["gen"])
     times, t_start = [], time.perf_counter()
@@ -491,6 +497,8 @@ def main():
     ap.add_argument("--window", type=int, default=0, help="override the workload's window (sweeps)")
     ap.add_argument("--inner", type=int, default=0, help="override the workload's inner iterations per step (sweeps)")
     ap.add_argument("--prefill-r", type=int, default=0, help="override the workload's prefill recurrence (profiling aid)")
+    ap.add_argument("--temperature", type=float, default=-1.0, help="override the workload's sampling temperature (sweeps)")
+    ap.add_argument("--top-p", type=float, default=0.0, help="top-p of Sample (sweeps; needs a temperature > 0)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

@@ -79,6 +79,12 @@ typedef struct {
                                   z <- (1 - b_t) z + b_t z_noise, b_t = beta max(0, 1 - t / T) at a
                                   position's step t; T = window (fixed exit) or
                                   ceil(max_iters_per_pos / inner_iters); 0 <= beta <= 1, 0 = off  */
+    float top_p;               /* Appendix (sampling settings of the evaluation: temperature 0.2,
+                                  top-p 0.95): with temperature > 0 and 0 < top_p < 1, Sample draws
+                                  from the most probable tokens up to the first at which the
+                                  cumulative probability under softmax(logits / temperature) reaches
+                                  top_p (equal logits at the cut stay together), renormalised;
+                                  0 or 1 = off.  Needs vocab <= 65536 (else INVALID_ARG)          */
 } rd_session_config;
 
 typedef struct {

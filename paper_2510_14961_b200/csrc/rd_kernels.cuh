@@ -543,6 +543,259 @@ sample_scan_kernel(const RowSource src, int vocab, int chunk, const int* __restr
     }
 }
 
+// Sample(p) with top-p (temperature > 0 and top_p < 1; the evaluation's settings in the paper's
+// Appendix are temperature 0.2, top-p 0.95), one kernel.  A cluster of NUC_CLUSTER blocks takes a
+// row; every thread keeps NUC_PER logits and their Gumbel-max scores in registers.  With M = max logit, mass_v = exp((l_v - M) / T), Z = sum of masses, the kept set is
+//   {v : l_v >= tau}, tau the largest value with mass{l_v >= tau} >= top_p Z
+// (the most probable tokens up to the first at which the cumulative probability reaches top_p, equal
+// logits at the cut kept together), and v is in it exactly when mass{l_w > l_v} < top_p Z.
+// The draft is the arg max of the scores over the kept set.  It is found without tau: take the arg
+// max c over the tokens still eligible (all, at first); if mass{l_w > l_c} < top_p Z it is the draft;
+// otherwise c and every token with a logit <= l_c are outside the kept set and leave the eligible
+// ones.  A try succeeds with the probability of the kept set (>= top_p), so NUC_TRIES tries almost
+// always do; the rows they leave undecided compute tau by a search over the order-preserving integer
+// image of float32 (NUC_CUTS thresholds per round) and take the arg max over {l_v >= tau}.
+// All sums are taken in a fixed order (thread, warp tree, warps of a block, blocks of the cluster by
+// rank), so every block takes the same decisions and the result is bit-reproducible.
+constexpr int NUC_CLUSTER = 8;
+constexpr int NUC_THREADS = 256;
+constexpr int NUC_PER = 32;                                   // logits per thread, as 8 quads
+constexpr int NUC_MAX_VOCAB = NUC_CLUSTER * NUC_THREADS * NUC_PER;   // 65536
+constexpr int NUC_TRIES = 4;
+constexpr int NUC_CUTS = 7;                                   // thresholds per round of the search for tau
+
+__device__ __forceinline__ uint32_t float_order_key(float x) {
+    const uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+struct NucShared {
+    float warp_f[NUC_THREADS / 32];
+    int warp_i[NUC_THREADS / 32];
+    uint32_t warp_k[NUC_THREADS / 32];
+    float sum_slots[2 * NUC_CLUSTER];                         // double-buffered: one cluster barrier per reduction
+    float arg_v[2 * NUC_CLUSTER];
+    int arg_i[2 * NUC_CLUSTER];
+    uint32_t arg_k[2 * NUC_CLUSTER];
+    float cut_part[(NUC_THREADS / 32) * NUC_CUTS];
+    float cut_slots[2 * NUC_CLUSTER * NUC_CUTS];
+};
+
+// Sum of `v` over the cluster, the same bits in every thread of every block.
+__device__ __forceinline__ float nuc_cluster_sum(float v, NucShared& sh, int& phase, cooperative_groups::cluster_group& cluster) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+    if ((threadIdx.x & 31) == 0) sh.warp_f[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < NUC_CLUSTER) {
+        float b = 0.f;
+        for (int w = 0; w < NUC_THREADS / 32; w++) b += sh.warp_f[w];
+        *cluster.map_shared_rank(&sh.sum_slots[phase * NUC_CLUSTER + blockIdx.x], threadIdx.x) = b;   // into every block's table
+    }
+    cluster.sync();
+    float tot = 0.f;
+    for (int k = 0; k < NUC_CLUSTER; k++) tot += sh.sum_slots[phase * NUC_CLUSTER + k];
+    phase ^= 1;
+    return tot;
+}
+
+// Arg max (lowest index on ties) over the cluster, with the winner's key; same result everywhere.
+__device__ __forceinline__ void nuc_cluster_argmax(float& best, int& bi, uint32_t& bk, NucShared& sh, int& phase,
+                                                   cooperative_groups::cluster_group& cluster) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, s);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, s);
+        const uint32_t ok = __shfl_xor_sync(0xffffffffu, bk, s);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; bk = ok; }
+    }
+    if ((threadIdx.x & 31) == 0) { sh.warp_f[threadIdx.x >> 5] = best; sh.warp_i[threadIdx.x >> 5] = bi; sh.warp_k[threadIdx.x >> 5] = bk; }
+    __syncthreads();
+    if (threadIdx.x < NUC_CLUSTER) {
+        float v = sh.warp_f[0]; int i = sh.warp_i[0]; uint32_t k = sh.warp_k[0];
+        for (int w = 1; w < NUC_THREADS / 32; w++)
+            if (sh.warp_f[w] > v || (sh.warp_f[w] == v && sh.warp_i[w] < i)) { v = sh.warp_f[w]; i = sh.warp_i[w]; k = sh.warp_k[w]; }
+        const int slot = phase * NUC_CLUSTER + blockIdx.x;
+        *cluster.map_shared_rank(&sh.arg_v[slot], threadIdx.x) = v;
+        *cluster.map_shared_rank(&sh.arg_i[slot], threadIdx.x) = i;
+        *cluster.map_shared_rank(&sh.arg_k[slot], threadIdx.x) = k;
+    }
+    cluster.sync();
+    best = -INFINITY; bi = 0x7fffffff; bk = 0;
+    for (int c = 0; c < NUC_CLUSTER; c++) {
+        const int slot = phase * NUC_CLUSTER + c;
+        if (sh.arg_v[slot] > best || (sh.arg_v[slot] == best && sh.arg_i[slot] < bi)) { best = sh.arg_v[slot]; bi = sh.arg_i[slot]; bk = sh.arg_k[slot]; }
+    }
+    phase ^= 1;
+}
+
+__global__ void __launch_bounds__(NUC_THREADS, 2)
+sample_nucleus_kernel(const RowSource src, int vocab, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                      float temperature, float top_p, uint64_t seed, float* __restrict__ logits_store,
+                      int* __restrict__ draft, int* __restrict__ tokens, int tok_stride) {
+    __shared__ NucShared sh;
+    pdl_enter();
+    cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+    const int r = blockIdx.y;
+    const int p = row_pos[r];
+    if (p < 0) return;                                         // the whole cluster leaves
+    cluster.sync();                                            // nobody writes into a block's tables before it runs
+
+    // quad q of the row belongs to thread (q mod 2048): consecutive threads read consecutive quads
+    float x[NUC_PER];
+#pragma unroll
+    for (int i = 0; i < NUC_PER / 4; i++) {
+        const int v = 4 * (i * (NUC_CLUSTER * NUC_THREADS) + blockIdx.x * NUC_THREADS + threadIdx.x);
+        if (v + 3 < vocab && (vocab & 3) == 0) {
+            const float4 q = row_source_load4(src, r, v);
+            x[4 * i] = q.x; x[4 * i + 1] = q.y; x[4 * i + 2] = q.z; x[4 * i + 3] = q.w;
+            if (logits_store) *reinterpret_cast<float4*>(logits_store + (size_t)r * vocab + v) = q;
+        } else {
+#pragma unroll
+            for (int a = 0; a < 4; a++) {
+                x[4 * i + a] = v + a < vocab ? row_source_load(src, r, v + a) : -INFINITY;
+                if (logits_store && v + a < vocab) logits_store[(size_t)r * vocab + v + a] = x[4 * i + a];
+            }
+        }
+    }
+    // Gumbel-max scores (same noise as sample_scan_kernel); -inf beyond the vocabulary
+    float sc[NUC_PER];
+    {
+        const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+        const uint32_t seq = (uint32_t)row_seq[r];
+#pragma unroll
+        for (int i = 0; i < NUC_PER / 4; i++) {
+            const int v = 4 * (i * (NUC_CLUSTER * NUC_THREADS) + blockIdx.x * NUC_THREADS + threadIdx.x);
+            const uint4 w4 = philox4x32_10(make_uint4((uint32_t)(v >> 2), (uint32_t)(p + 1), seq, STREAM_GUMBEL), key);
+            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int a = 0; a < 4; a++) {
+                const float g = -logf(-logf(unit_open(w[a])));
+                sc[4 * i + a] = v + a < vocab ? __fadd_rn(__fdiv_rn(x[4 * i + a], temperature), g) : -INFINITY;
+            }
+        }
+    }
+    int phase = 0;
+    // M: max over the cluster (exact, so the order does not matter)
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < NUC_PER; j++) mx = fmaxf(mx, x[j]);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+    if ((threadIdx.x & 31) == 0) sh.warp_f[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x < NUC_CLUSTER) {
+        float b = -INFINITY;
+        for (int w = 0; w < NUC_THREADS / 32; w++) b = fmaxf(b, sh.warp_f[w]);
+        *cluster.map_shared_rank(&sh.sum_slots[phase * NUC_CLUSTER + blockIdx.x], threadIdx.x) = b;
+    }
+    cluster.sync();
+    float M = -INFINITY;
+    for (int k = 0; k < NUC_CLUSTER; k++) M = fmaxf(M, sh.sum_slots[phase * NUC_CLUSTER + k]);
+    phase ^= 1;
+
+    int token = 0x7fffffff;
+    uint32_t allow = 0;                                        // eligible: keys >= allow
+    if (M > -INFINITY && M < INFINITY) {
+        const float c = 1.4426950408889634f / temperature;    // exp(d / T) = 2^(d c)
+        // masses are recomputed where they are used (the same bits every time): two blocks fit an SM
+        auto mass_of = [&](float l) { return l > -INFINITY ? exp2f((l - M) * c) : 0.f; };
+        float zs = 0.f;
+#pragma unroll
+        for (int j = 0; j < NUC_PER; j++) zs += mass_of(x[j]);
+        const float Z = nuc_cluster_sum(zs, sh, phase, cluster);
+        const float target = top_p * Z;
+        bool undecided = true;
+        for (int t = 0; t < NUC_TRIES; t++) {
+            float best = -INFINITY;
+            int bi = 0x7fffffff;
+            uint32_t bk = 0;
+#pragma unroll
+            for (int j = 0; j < NUC_PER; j++) {
+                const int v = 4 * ((j >> 2) * (NUC_CLUSTER * NUC_THREADS) + blockIdx.x * NUC_THREADS + threadIdx.x) + (j & 3);
+                const uint32_t k = float_order_key(x[j]);
+                if (k >= allow && (sc[j] > best || (sc[j] == best && v < bi))) { best = sc[j]; bi = v; bk = k; }
+            }
+            nuc_cluster_argmax(best, bi, bk, sh, phase, cluster);
+            if (bi == 0x7fffffff) break;                       // nothing eligible (a row of NaN)
+            float above = 0.f;
+#pragma unroll
+            for (int j = 0; j < NUC_PER; j++) above += float_order_key(x[j]) > bk ? mass_of(x[j]) : 0.f;
+            above = nuc_cluster_sum(above, sh, phase, cluster);
+            if (above < target) { token = bi; undecided = false; break; }
+            allow = bk + 1;                                    // bk is a finite number's key: no wrap
+        }
+        if (undecided) {
+            // tau: largest key t with mass{key_v >= t} >= target; at t = 0 the mass is Z, above key(M) it is 0.
+            // Each round cuts [lo, hi) at up to NUC_CUTS thresholds and sums the mass above each of them.
+            uint32_t lo = 0, hi = float_order_key(M);
+            if (hi != 0xffffffffu) hi += 1;
+            while (hi - lo > 1) {
+                const uint32_t span = hi - lo;
+                const uint32_t step = (uint32_t)(((uint64_t)span + NUC_CUTS) / (NUC_CUTS + 1));   // ceil(span / (cuts + 1)) >= 1
+                // thresholds lo + (i + 1) step below hi; at least one since span >= 2
+                const int nt = (int)min((uint64_t)NUC_CUTS, ((uint64_t)span - 1) / step);
+                float acc[NUC_CUTS];
+                uint32_t cut[NUC_CUTS];                        // unused thresholds: above every key of a number
+#pragma unroll
+                for (int i = 0; i < NUC_CUTS; i++) {
+                    acc[i] = 0.f;
+                    cut[i] = i < nt ? lo + (uint32_t)(i + 1) * step : 0xffffffffu;
+                }
+#pragma unroll
+                for (int j = 0; j < NUC_PER; j++) {
+                    const uint32_t k = float_order_key(x[j]);
+                    const float mj = mass_of(x[j]);
+#pragma unroll
+                    for (int i = 0; i < NUC_CUTS; i++) acc[i] += k >= cut[i] ? mj : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < NUC_CUTS; i++) {
+#pragma unroll
+                    for (int sft = 16; sft > 0; sft >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], sft);
+                    if ((threadIdx.x & 31) == 0) sh.cut_part[(threadIdx.x >> 5) * NUC_CUTS + i] = acc[i];
+                }
+                __syncthreads();
+                if (threadIdx.x < NUC_CUTS) {
+                    float b = 0.f;
+                    for (int w = 0; w < NUC_THREADS / 32; w++) b += sh.cut_part[w * NUC_CUTS + threadIdx.x];
+                    for (int k = 0; k < NUC_CLUSTER; k++)      // every block's table gets this block's sums
+                        *cluster.map_shared_rank(&sh.cut_slots[(phase * NUC_CLUSTER + blockIdx.x) * NUC_CUTS + threadIdx.x], k) = b;
+                }
+                cluster.sync();
+                int count = 0;                                 // thresholds whose mass still reaches the target
+                for (int i = 0; i < nt; i++) {
+                    float tot = 0.f;
+                    for (int k = 0; k < NUC_CLUSTER; k++) tot += sh.cut_slots[(phase * NUC_CLUSTER + k) * NUC_CUTS + i];
+                    if (tot >= target) count = i + 1; else break;
+                }
+                phase ^= 1;
+                const uint32_t new_lo = count ? lo + (uint32_t)count * step : lo;
+                if (count < nt) hi = lo + (uint32_t)(count + 1) * step;
+                lo = new_lo;
+            }
+            allow = max(allow, lo);                            // tokens the tries removed are below tau anyway
+        }
+    }
+    if (token == 0x7fffffff) {
+        // arg max over the eligible tokens (the kept set after the search; everything for a row of NaN)
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
+        uint32_t bk = 0;
+#pragma unroll
+        for (int j = 0; j < NUC_PER; j++) {
+            const int v = 4 * ((j >> 2) * (NUC_CLUSTER * NUC_THREADS) + blockIdx.x * NUC_THREADS + threadIdx.x) + (j & 3);
+            if (float_order_key(x[j]) >= allow && (sc[j] > best || (sc[j] == best && v < bi))) { best = sc[j]; bi = v; bk = 1; }
+        }
+        nuc_cluster_argmax(best, bi, bk, sh, phase, cluster);
+        token = bi == 0x7fffffff ? 0 : bi;                     // all -inf / NaN row: defined result
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        draft[r] = token;
+        tokens[(size_t)row_seq[r] * tok_stride + p + 1] = token;
+    }
+}
+
 // Second kernel, one thread per row: best of the chunks (lowest index on ties) -> draft.
 __global__ void sample_pick_kernel(const float* __restrict__ best_val, const int* __restrict__ best_idx, int n_chunks,
                                    int n_rows, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
@@ -584,7 +837,7 @@ delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int 
 }
 
 // End of a step, one thread per sequence: count the step on every in-flight row, find k* (the
-// longest finished prefix; Eq. 3 / Algorithm 1 line 14), commit, drop, append one fresh row while
+// longest finished prefix; Eq. 3 and the freeze step of Algorithm 1), commit, drop, append one fresh row while
 // the wavefront is below `window` and the row's draft is still wanted.
 struct SeqState {
     int* n_prompt; int* n_committed; int* win_len; int* done;

@@ -332,6 +332,9 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     if (sc.batch < 1 || sc.max_context < 2 || sc.max_window < 1 || sc.max_new_tokens < 0) return RD_E_INVALID_ARG;
     if (sc.max_iters_per_pos < 1 || !(sc.temperature >= 0.f)) return RD_E_INVALID_ARG;
     if (!(sc.eta >= 0.f && sc.eta < 1.f) || !(sc.beta >= 0.f && sc.beta <= 1.f)) return RD_E_INVALID_ARG;
+    if (!(sc.top_p >= 0.f && sc.top_p <= 1.f)) return RD_E_INVALID_ARG;
+    // the top-p kernel keeps a row's logits in the registers of one cluster
+    if (sc.temperature > 0.f && sc.top_p > 0.f && sc.top_p < 1.f && m->cfg.vocab > NUC_MAX_VOCAB) return RD_E_INVALID_ARG;
     if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
     rd_session* s = new (std::nothrow) rd_session();
     if (!s) return RD_E_OOM;
@@ -679,6 +682,12 @@ template <typename T> struct Eng {
         RD_TRY(norm<T>(s, x, nullptr, s->m->g_final, (T*)s->act_h, n_rows));
         RowSource lg;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, n_rows, &lg));
+        if (s->sc.temperature > 0.f && s->sc.top_p > 0.f && s->sc.top_p < 1.f) {
+            LAUNCH_CLUSTER(s, sample_nucleus_kernel, (NUC_CLUSTER, n_rows), NUC_THREADS, 0, NUC_CLUSTER, lg, c.vocab, s->row_pos,
+                           s->row_seq, s->sc.temperature, s->sc.top_p, s->sc.seed, s->sc.keep_logits ? s->logits : (float*)nullptr,
+                           s->draft, s->tokens, s->tok_stride);
+            return RD_OK;
+        }
         // vocabulary split into at most SAMPLE_CHUNKS runs (multiples of 4) per row
         const int chunk = ((c.vocab + SAMPLE_CHUNKS - 1) / SAMPLE_CHUNKS + 3) / 4 * 4;
         const int n_chunks = (c.vocab + chunk - 1) / chunk;

@@ -31,10 +31,15 @@ class LockStep:
 
     A draft mismatch is admissible only when the oracle's own top-2 gap (of the scores that decide
     the token) is below `tie_gap`; the oracle then follows the GPU's token so that both continue
-    from the same y_current.  The fp32 configuration uses tie_gap = 0: any mismatch fails."""
+    from the same y_current.  The fp32 configuration uses tie_gap = 0: any mismatch fails.
+
+    With top-p sampling a token whose membership of the kept set hangs on the tolerance of the logits
+    may legitimately differ: with u(v) the probability mass (oracle logits) of the tokens strictly
+    more probable than v, the GPU's token g is admissible when u(g) < top_p + nucleus_band and no
+    token w with u(w) < top_p - nucleus_band beats g's score by more than tie_gap."""
 
     def __init__(self, sampler: orc.Sampler, session: rd.Session, seqs, tol: Tolerance, tie_gap=0.0,
-                 check_logits=True, logit_noise=None):
+                 check_logits=True, logit_noise=None, nucleus_band=0.0):
         """logit_noise = (rms, fraction, max_abs): instead of bounding every logit by `tol`, bound the
         rms error, the fraction of logits outside `tol` and the largest error (used at the full
         3.5B widths, where bf16 rounding noise amplified by the random-init layers puts a few
@@ -42,7 +47,9 @@ class LockStep:
         self.sm, self.sess, self.seqs, self.tol, self.tie_gap = sampler, session, seqs, tol, tie_gap
         self.check_logits = check_logits
         self.logit_noise = logit_noise
+        self.nucleus_band = nucleus_band
         self.near_ties = 0
+        self.boundary_cases = 0
         self.n_drafts = 0
         self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0}
         self.steps = 0
@@ -53,6 +60,16 @@ class LockStep:
             return l32
         return l32 / np.float32(self.sm.temperature) + orc.gumbel_noise(self.sm.seed, sq.seq_id, token_pos,
                                                                         l32.shape[0])
+
+    def _upper_mass(self, logits):
+        """u(v): probability (softmax(l / T), float64) of the tokens with a logit strictly above l_v."""
+        l = logits.astype(np.float32).astype(np.float64)
+        q = np.exp((l - l.max()) / float(self.sm.temperature))
+        q /= q.sum()
+        vals, inv = np.unique(l, return_inverse=True)            # ascending
+        mass_of_val = np.bincount(inv, weights=q, minlength=len(vals))
+        above = np.concatenate([np.cumsum(mass_of_val[::-1])[::-1][1:], [0.0]])
+        return above[inv]
 
     def compare(self, infos, delta_checked=True):
         self.steps += 1
@@ -90,9 +107,21 @@ class LockStep:
                 if drafts[i] == info["drafts"][i]:
                     continue
                 sc = self._scores(info["logits"][i], sq, int(info["pos"][i]) + 1)
-                gap = float(sc[info["drafts"][i]] - sc[drafts[i]])
-                assert 0 <= gap <= self.tie_gap, \
-                    f"step {self.steps} seq {b} row {i}: GPU token {drafts[i]} vs oracle {info['drafts'][i]}, gap {gap:.3e}"
+                top_p = getattr(self.sm, "top_p", 1.0)
+                if self.sm.temperature > 0 and top_p < 1.0:
+                    u = self._upper_mass(info["logits"][i])
+                    g = int(drafts[i])
+                    sure = u < top_p - self.nucleus_band
+                    assert u[g] < top_p + self.nucleus_band, \
+                        f"step {self.steps} seq {b} row {i}: GPU token {g} outside the nucleus (mass above it {u[g]:.4f})"
+                    lead = float(sc[sure].max() - sc[g]) if sure.any() else 0.0
+                    assert lead <= self.tie_gap, \
+                        f"step {self.steps} seq {b} row {i}: GPU token {g} vs oracle {info['drafts'][i]}, beaten by {lead:.3e}"
+                    self.boundary_cases += 1
+                else:
+                    gap = float(sc[info["drafts"][i]] - sc[drafts[i]])
+                    assert 0 <= gap <= self.tie_gap, \
+                        f"step {self.steps} seq {b} row {i}: GPU token {drafts[i]} vs oracle {info['drafts'][i]}, gap {gap:.3e}"
                 self.near_ties += 1
                 self.sm.force_draft(sq, int(info["pos"][i]) + 1, int(drafts[i]))
             ncom, done = self.sess.committed(b)
