@@ -122,7 +122,7 @@ __device__ __forceinline__ void normal4(uint4 x, float sigma, float* out) {
     }
 }
 
-// Start of a pass over the rows.
+// Start of a pass over the rows; grid (rows, parts).
 // s_0 ~ N(0, sigma^2 I), keyed by (seed, sequence, position): element j is output j%4 of block j/4.
 // only_fresh: only rows whose step counter is 0 (rows appended last step) get s_0; the others keep z.
 // With z_prev the kernel also takes the snapshot z_prev <- z of every active row (Algorithm 2).
@@ -143,10 +143,14 @@ __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const uint32_t seq = (uint32_t)row_seq[r];
     const int nb = (hidden + 3) / 4;
-    for (int blk = threadIdx.x; blk < nb; blk += blockDim.x) {
+    const bool vec = (hidden & 3) == 0 && (ldz & 3) == 0;       // 16-byte accesses
+    for (int blk = blockIdx.y * blockDim.x + threadIdx.x; blk < nb; blk += gridDim.y * blockDim.x) {
         float v[4];
         if (fresh) {
             normal4(philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, seq, STREAM_INIT_STATE), key), sigma, v);
+        } else if (vec) {
+            const float4 q = *reinterpret_cast<const float4*>(z + (size_t)r * ldz + blk * 4);
+            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         } else {
 #pragma unroll
             for (int a = 0; a < 4; a++) v[a] = blk * 4 + a < hidden ? z[(size_t)r * ldz + blk * 4 + a] : 0.f;
@@ -157,6 +161,11 @@ __global__ void init_state_kernel(const int* __restrict__ row_pos, const int* __
             normal4(philox4x32_10(make_uint4((uint32_t)blk, (uint32_t)p, seq, STREAM_NOISE | ((uint32_t)t << 8)), key), sigma, nz);
 #pragma unroll
             for (int a = 0; a < 4; a++) zn[a] = __fadd_rn(__fmul_rn(1.0f - b, v[a]), __fmul_rn(b, nz[a]));
+        }
+        if (vec) {
+            if (fresh || b > 0.f) *reinterpret_cast<float4*>(z + (size_t)r * ldz + blk * 4) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+            if (z_prev) *reinterpret_cast<float4*>(z_prev + (size_t)r * ldz + blk * 4) = make_float4(v[0], v[1], v[2], v[3]);
+            continue;
         }
 #pragma unroll
         for (int a = 0; a < 4; a++)
@@ -818,7 +827,8 @@ __global__ void sample_pick_kernel(const float* __restrict__ best_val, const int
 }
 
 // delta_i = ||z_i - z_prev,i|| / ||z_i||  (Eq. 3); +inf when ||z_i|| = 0.
-__global__ void __launch_bounds__(256)
+constexpr int DELTA_THREADS = 1024;              // a 5280-wide row is one 16-byte load per thread and array
+__global__ void __launch_bounds__(DELTA_THREADS)
 delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int hidden,
              const int* __restrict__ row_pos, float* __restrict__ delta) {
     pdl_enter();
@@ -826,10 +836,25 @@ delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int 
     const int r = blockIdx.x;
     if (row_pos[r] < 0) return;
     float num = 0.f, den = 0.f;
-    for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
-        const float a = z[(size_t)r * hidden + j], d = a - z_prev[(size_t)r * hidden + j];
-        num += d * d;
-        den += a * a;
+    if ((hidden & 3) == 0) {
+        const float4* a4 = reinterpret_cast<const float4*>(z + (size_t)r * hidden);
+        const float4* b4 = reinterpret_cast<const float4*>(z_prev + (size_t)r * hidden);
+        for (int j = threadIdx.x; j < hidden / 4; j += blockDim.x) {
+            const float4 a = a4[j], b = b4[j];
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const float d = av[k] - bv[k];
+                num += d * d;
+                den += av[k] * av[k];
+            }
+        }
+    } else {
+        for (int j = threadIdx.x; j < hidden; j += blockDim.x) {
+            const float a = z[(size_t)r * hidden + j], d = a - z_prev[(size_t)r * hidden + j];
+            num += d * d;
+            den += a * a;
+        }
     }
     num = block_sum(num, sm);
     den = block_sum(den, sm);

@@ -497,6 +497,9 @@ static Pending plain_rows(const float* x, size_t ld) {
     return p;
 }
 
+// blocks of 128 threads per row of init_state_kernel: one 4-element group per thread, at most 16
+static int init_parts(int hidden) { return std::max(1, std::min(16, ((hidden + 3) / 4 + 127) / 128)); }
+
 template <typename T> struct Eng {
     static bool tc_usable(const rd_session* s, const TcAct* ta, const TcWeight* tw) {
         return sizeof(T) == 2 && s->gemm_path >= 1 && ta && tw && ta->valid && tw->valid;
@@ -719,12 +722,12 @@ template <typename T> struct Eng {
         // (stabilisers of Section 3.4 apply to sampler steps, not to the sequential decoder)
         const float eta = stabilise ? s->sc.eta : 0.f, beta = stabilise ? s->sc.beta : 0.f;
         const int sched = eps <= 0.f ? window : (s->sc.max_iters_per_pos + inner - 1) / inner;
-        LAUNCH(s, init_state_kernel, n, 128, 0, s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma, s->sc.seed, s->z,
+        LAUNCH(s, init_state_kernel, dim3(n, init_parts(h)), 128, 0, s->row_pos, s->row_seq, s->row_steps, 1, h, c.init_sigma, s->sc.seed, s->z,
                (size_t)h, s->z_prev, beta, sched);
         RD_TRY(prelude(s, n, s->e, eta));
         for (int j = 0; j < inner; j++) RD_TRY(core(s, s->e, s->z, s->z, n));
         RD_TRY(coda(s, s->z, n, true));
-        LAUNCH(s, delta_kernel, n, 256, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
+        LAUNCH(s, delta_kernel, n, DELTA_THREADS, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
         SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
         LAUNCH(s, advance_kernel, (B + 63) / 64, 64, 0, st, s->delta, B, s->sc.max_window, window, inner, eps,
                s->sc.max_iters_per_pos, s->sc.max_new_tokens);
@@ -747,7 +750,7 @@ template <typename T> struct Eng {
                 float* zc = s_all + (size_t)c0 * h;
                 if (pass == 0) {
                     RD_TRY(prelude(s, nr, ec));
-                    LAUNCH(s, init_state_kernel, nr, 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
+                    LAUNCH(s, init_state_kernel, dim3(nr, init_parts(h)), 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
                            s->sc.seed, zc, (size_t)h, (float*)nullptr, 0.f, 1);
                 } else if (pass <= r) {
                     RD_TRY(core(s, ec, zc, zc, nr));
