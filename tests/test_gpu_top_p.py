@@ -52,6 +52,36 @@ def test_fp32_lock_step_with_top_p(temperature, top_p):
     assert differs > 0
 
 
+@pytest.mark.parametrize("vocab", [65536, 50001])
+def test_full_vocabulary_and_ragged_vocabulary(vocab):
+    """The largest vocabulary the top-p kernel takes (every thread of the row's cluster holds its full
+    32 logits) and one that is not a multiple of 4 (scalar loads, a partly filled last group)."""
+    shape = dict(SMALL, vocab=vocab, n_core=1)
+    sess, sm = _pair(shape, 3, 6, 1.0, 0.9, batch=2, std=0.1)
+    seqs = _prefill(sm, sess, shape, [4, 7], 1, 6)
+    ls = LockStep(sm, sess, seqs, Tolerance(1e-4), nucleus_band=1e-3)
+    while not ls.all_done():
+        ls.df(3, 1, 0.0)
+    ls.final_tokens_equal()
+    assert ls.boundary_cases <= 1
+    # and with a cut so low that most rows go through the search for tau
+    sess, sm = _pair(shape, 3, 6, 1.0, 0.002, batch=2, std=0.1)
+    seqs = _prefill(sm, sess, shape, [4, 7], 1, 6)
+    ls = LockStep(sm, sess, seqs, Tolerance(1e-4), nucleus_band=1e-5)
+    while not ls.all_done():
+        ls.df(3, 1, 0.0)
+    ls.final_tokens_equal()
+
+
+def test_vocabulary_beyond_the_kernel_limit_is_refused():
+    shape = dict(SMALL, vocab=65540, n_core=1)
+    model, w = make_oracle(shape, seed=0, std=0.1)
+    gm = gpu_model(shape, w)
+    with pytest.raises(rd.RdError):
+        rd.Session(gm, batch=1, max_context=64, max_window=2, max_new_tokens=4, temperature=1.0, top_p=0.9)
+    rd.Session(gm, batch=1, max_context=64, max_window=2, max_new_tokens=4, temperature=1.0).close()   # fine without top-p
+
+
 def test_bf16_twin_ragged_batch_top_p():
     """bf16 configuration (tensor-core GEMMs), ragged batch, adaptive exit, T = 1, top-p 0.9.  The
     logit tolerance moves the cumulative masses near the cut by a few percent: band 0.1."""
