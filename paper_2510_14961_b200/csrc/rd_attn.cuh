@@ -64,9 +64,17 @@ template <int D> struct AttCfg {
 // (groups of up to 64 rows).  KW = 32, for groups of at most 32 rows: warps 0,1 take the two query
 // blocks on the tile's first 32 keys, warps 2,3 the same queries on its last 32, and the two halves
 // are merged (first half, then second) through shared memory before the cluster merge.
+// Groups in the order the hardware should start them (blockIdx.z counts through it): the host
+// puts the longest contexts first so that the blocks that run longest do not start last.
+constexpr int ATT_MAX_ORDERED = 64;
+struct GroupOrder {
+    unsigned char idx[ATT_MAX_ORDERED];
+    int n;                              // 0: groups in index order
+};
+
 template <int D, int KW>
 __global__ void __launch_bounds__(128)
-attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
+attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
                    const int* __restrict__ row_seq, int rows_per_group, int n_rows,
                    const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
                    size_t head_stride, int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
@@ -81,7 +89,7 @@ attn_window_kernel(const __nv_bfloat16* __restrict__ q_t, const int* __restrict_
     pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sp = blockIdx.x, n_splits = gridDim.x, hd = blockIdx.y;
-    const int r0 = blockIdx.z * rows_per_group;
+    const int r0 = (order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z) * rows_per_group;
     const int nq = min(rows_per_group, n_rows - r0);
     // positions of the group's rows; kv_len = 1 + the largest of them
     __shared__ int warp_max[4];

@@ -247,6 +247,7 @@ struct rd_session {
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
+    std::vector<int> grp_ctx;   // the same bound per attention group (sequence in decode, row block in prefill)
     int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128)
     void *act_h = nullptr, *act_2h = nullptr, *act_i = nullptr, *q_t = nullptr;
     void *Kc[3] = {nullptr, nullptr, nullptr}, *Vc[3] = {nullptr, nullptr, nullptr};
@@ -567,7 +568,17 @@ template <typename T> struct Eng {
         int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
         ns = std::max(1, std::min(std::min(ns, 8), tiles));
         const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
-        LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW>), (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, (const bf16*)s->q_t,
+        // longest contexts first (s->grp_ctx: the host's bound of each group's context)
+        GroupOrder order;
+        order.n = 0;
+        if (groups > 1 && groups <= ATT_MAX_ORDERED && (int)s->grp_ctx.size() >= groups) {
+            int ids[ATT_MAX_ORDERED];
+            for (int g = 0; g < groups; g++) ids[g] = g;
+            std::stable_sort(ids, ids + groups, [&](int a, int b) { return s->grp_ctx[a] > s->grp_ctx[b]; });
+            for (int g = 0; g < groups; g++) order.idx[g] = (unsigned char)ids[g];
+            order.n = groups;
+        }
+        LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW>), (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, order, (const bf16*)s->q_t,
                        s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
                        (bf16*)s->act_h);
         return RD_OK;
@@ -709,12 +720,14 @@ template <typename T> struct Eng {
         s->ctx_total = 0;
         s->ctx_max = 1;
         s->grp_rows = s->sc.max_window;
+        s->grp_ctx.assign(B, 0);
         for (int b = 0; b < B; b++)
             if (s->prefilled[b]) {
                 s->host_steps[b]++;
                 const int ctx = std::min(s->host_prompt_len[b] + s->host_steps[b], s->host_prompt_len[b] + s->sc.max_new_tokens);
                 s->ctx_total += ctx;
                 s->ctx_max = std::max(s->ctx_max, ctx);
+                s->grp_ctx[b] = ctx;
             }
         LAUNCH(s, plan_rows_kernel, (n + 127) / 128, 128, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window,
                s->row_pos, s->row_seq, s->step_first, s->step_n);
@@ -745,6 +758,8 @@ template <typename T> struct Eng {
                 s->grp_rows = ATT_QMAX;
                 s->ctx_max = c0 + nr;
                 s->ctx_total = c0 + nr;
+                s->grp_ctx.clear();
+                for (int g0 = 0; g0 < nr; g0 += ATT_QMAX) s->grp_ctx.push_back(c0 + std::min(nr, g0 + ATT_QMAX));
                 LAUNCH(s, fill_rows_kernel, (s->R + 127) / 128, 128, 0, seq, c0, nr, s->R, s->row_pos, s->row_seq);
                 float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
                 float* zc = s_all + (size_t)c0 * h;
