@@ -219,8 +219,8 @@ int rd_profile_enable(rd_session* s, int32_t on);
 int rd_profile_read(rd_session* s, rd_profile_t* out);
 
 /* rd_set_gemm_path -- 0: SIMT kernels everywhere; 1 (default for RD_BF16): tcgen05 tensor-core
- * GEMMs where the shape allows, tiles of 256 rows on CTA pairs (one MMA of 256 features over two
- * SMs); 2: as 1 with the 256-row tiles on single CTAs.  For measurement and parity tests. */
+ * GEMMs where the shape allows, tiles of 128 and 256 rows on CTA pairs (one MMA of 256 features over
+ * two SMs); 2: as 1 with those tiles on single CTAs.  For measurement and parity tests. */
 int rd_set_gemm_path(rd_session* s, int32_t path);
 
 /* rd_set_launch_chaining -- 1 (default): the kernels of a step are launched as a programmatic-

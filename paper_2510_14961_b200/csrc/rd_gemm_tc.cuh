@@ -30,7 +30,7 @@
 // do not depend on earlier kernels), and only then waits for the predecessor before touching
 // activations or the scratch buffer.
 //
-// Tiles of 256 rows run on CTA pairs (gemm_tc_pair_kernel, tcgen05 cta_group::2): the two CTAs of a
+// Tiles of 128 and 256 rows run on CTA pairs (gemm_tc_pair_kernel, tcgen05 cta_group::2): the two CTAs of a
 // cluster each stage one 128-feature weight tile and half of the rows, and one MMA of M = 256 spans
 // both SMs.  Same units, slots and consumers.
 //
@@ -468,10 +468,10 @@ struct UnitCursor {
 };
 
 // ---------------------------------------------------------------------------------------------
-// 256-row tiles on a CTA pair.  Two CTAs of a cluster (one per SM of a pair) share every unit: a unit
-// is (256 output features, 256 rows, one k-block); CTA `rank` loads the rank-th 128-feature weight
-// tile and the rank-th 128 rows of the activation tile, the leader (rank 0) issues one MMA of
-// M = 256, N = 256 per K = 16 slice, and each CTA's TMEM receives its own 128 features x 256 rows.
+// 128- and 256-row tiles on a CTA pair.  Two CTAs of a cluster (one per SM of a pair) share every unit: a
+// unit is (256 output features, BN rows, one k-block); CTA `rank` loads the rank-th 128-feature weight
+// tile and the rank-th half of the rows of the activation tile, the leader (rank 0) issues one MMA of
+// M = 256, N = BN per K = 16 slice, and each CTA's TMEM receives its own 128 features x BN rows.
 // Against one CTA running two M = 128 MMAs over a full 256-row activation tile, each SM stages half
 // the activation bytes per weight byte (32 KB instead of 48 KB of shared-memory writes per k-block and
 // each half of the activation tile is read from shared memory once for both tensor cores), and the ring is 6 deep.
@@ -482,21 +482,22 @@ struct UnitCursor {
 //   acc_empty[b]  leader's, 8 arrivals: the four TMEM-reading warps of both CTAs
 // Slots, segments and the consumer side are those of gemm_tc_kernel<256>, with a pair in place of a CTA.
 // ---------------------------------------------------------------------------------------------
-struct TcPairCfg {
-    static constexpr int BN = 256;                                    // rows of a unit (UMMA N)
+template <int BN_> struct TcPairCfg {
+    static constexpr int BN = BN_;                                    // rows of a unit (UMMA N): 128 or 256
     static constexpr int A_BYTES = TC_BM * TC_BK * 2;                 // this CTA's weight tile, 16 KB
-    static constexpr int B_BYTES = (BN / 2) * TC_BK * 2;              // this CTA's half of the rows, 16 KB
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = 6;
+    static constexpr int B_BYTES = (BN / 2) * TC_BK * 2;              // this CTA's half of the rows
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;             // 32 KB / 24 KB
+    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;         // 6 / 8
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int ACC_COLS = BN;
     static constexpr int NBUF = 2;
-    static constexpr int TMEM_COLS = NBUF * ACC_COLS;                 // 512: all of TMEM, one CTA per SM
+    static constexpr int TMEM_COLS = NBUF * ACC_COLS;                 // 512 / 256; one CTA per SM
 };
 
+template <int BN>
 __global__ void __launch_bounds__(TC_THREADS)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, const TcParams p) {
-    using C = TcPairCfg;
+    using C = TcPairCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* full = (uint64_t*)(smem + C::STAGES * C::STAGE_BYTES);
@@ -658,19 +659,22 @@ static inline int tc_pick_bn(int n_rows) { return n_rows <= 16 ? 0 : n_rows <= 3
 
 struct TcPlan {
     int bn_idx, bn, mt, kb, n_tiles_m, n_tiles_n, per, grid, max_seg;
+    bool pair;
     long long units;
     size_t scratch_elems;
 };
 // Every CTA gets `per` consecutive units (the last ones possibly fewer).
-// `pair`: 256-row tiles go to CTA pairs (gemm_tc_pair_kernel) instead of single CTAs.
+// `pair`: tiles of 128 and 256 rows go to CTA pairs (gemm_tc_pair_kernel) instead of single CTAs.
+constexpr int TC_PAIR_MIN_BN = 128;
 static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair = true) {
     TcPlan pl;
     pl.bn_idx = tc_pick_bn(n_rows);
     pl.bn = 16 << pl.bn_idx;
-    if (pl.bn <= RD_TC_2CTA_MAX_BN) n_sms *= TC_CTAS_PER_SM;
-    else if (pair) n_sms /= 2;                          // a CTA pair per two SMs takes a share
+    pl.pair = pair && pl.bn >= TC_PAIR_MIN_BN;
+    if (pl.pair) n_sms /= 2;                            // a CTA pair per two SMs takes a share
+    else if (pl.bn <= RD_TC_2CTA_MAX_BN) n_sms *= TC_CTAS_PER_SM;
     pl.kb = (K + TC_BK - 1) / TC_BK;
-    pl.mt = pl.bn == 256 ? 2 : 1;                       // = TcTiles<bn>::MT
+    pl.mt = pl.pair || pl.bn == 256 ? 2 : 1;            // feature tiles per unit (= TcTiles<bn>::MT for single CTAs)
     pl.n_tiles_m = (n_out + pl.mt * TC_BM - 1) / (pl.mt * TC_BM);   // units cover mt feature tiles
     pl.n_tiles_n = (n_rows + pl.bn - 1) / pl.bn;
     pl.units = (long long)pl.n_tiles_m * pl.n_tiles_n * pl.kb;
@@ -694,14 +698,15 @@ static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& 
                ? RD_OK : RD_E_CUDA;
 }
 
+template <int BN>
 static int tc_launch_pair(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, int pairs, bool chained) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TcPairCfg::SMEM) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcPairCfg<BN>::SMEM) != cudaSuccess)
             return RD_E_CUDA;
         attr_set = true;
     }
-    return launch_chained_cluster(gemm_tc_pair_kernel, dim3(2 * pairs), dim3(TC_THREADS), TcPairCfg::SMEM, st, chained, 2, mw, mx, p) ==
+    return launch_chained_cluster(gemm_tc_pair_kernel<BN>, dim3(2 * pairs), dim3(TC_THREADS), TcPairCfg<BN>::SMEM, st, chained, 2, mw, mx, p) ==
                    cudaSuccess ? RD_OK : RD_E_CUDA;
 }
 
@@ -722,9 +727,11 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
         case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);
         case 1: return tc_launch<32>(st, tw.map, ta.map[1], p, pl.grid, chained);
         case 2: return tc_launch<64>(st, tw.map, ta.map[2], p, pl.grid, chained);
-        case 3: return tc_launch<128>(st, tw.map, ta.map[3], p, pl.grid, chained);
+        case 3:
+            if (pl.pair) return tc_launch_pair<128>(st, tw.map, ta.map[2], p, pl.grid, chained);   // 64 rows per CTA
+            return tc_launch<128>(st, tw.map, ta.map[3], p, pl.grid, chained);
         default:
-            if (pair) return tc_launch_pair(st, tw.map, ta.map[3], p, pl.grid, chained);
+            if (pl.pair) return tc_launch_pair<256>(st, tw.map, ta.map[3], p, pl.grid, chained);   // 128 rows per CTA
             return tc_launch<256>(st, tw.map2, ta.map[4], p, pl.grid, chained);
     }
 }

@@ -141,6 +141,23 @@ def test_twin_window_64_rows():
 
 
 @pytest.mark.parametrize("path", [1, 2])
+def test_twin_batch_8_window_16_is_128_rows(path):
+    """128 rows in flight: the 128-row GEMM tile (path 1: on CTA pairs, 64 rows per CTA; path 2: single
+    CTAs), ragged prompts of up to 100 tokens (prefill chunks of 128 rows too), greedy, fixed exit."""
+    lens = rd_inputs.make_prompt_lengths(8, 3, 100, seed=4)
+    # (a row lives 16 steps here: the weaker feedback keeps rounding noise from growing along the recurrence)
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 16, 20, batch=8, cap=8, max_ctx=160, gemm_path=path, adapter_s_scale=0.25)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 2, 20)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    for _ in range(22):
+        if ls.all_done():
+            break
+        ls.df(16, 1, 0.0)
+    assert _ties_ok(ls)
+    assert sess.stats()["tc_gemm_launches"] > 0
+
+
+@pytest.mark.parametrize("path", [1, 2])
 def test_twin_batch_16_window_16_is_256_rows(path):
     """The batched-serving row count: 16 sequences x 16 in-flight rows = the 256-row GEMM tile (path 1:
     on CTA pairs, one MMA of 256 features over two SMs; path 2: on single CTAs), ragged prompts,
