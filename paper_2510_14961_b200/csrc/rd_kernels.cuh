@@ -221,16 +221,22 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
         const int j = m0 + threadIdx.x + i * blockDim.x;
         gr[i] = j < m1 ? g[j] : 0.f;
     }
+    const int r = blockIdx.y;
+    // where this thread's first group of four sits in the GEMM's scratch: arithmetic only, also before the wait
+    constexpr int NQ = 4;
+    const int m_first = m0 + threadIdx.x * 4;
+    RowSlots<NQ> first_slots;
+    first_slots.n = NQ + 1;
+    if (m_first < m1) first_slots = row_source_locate<NQ>(src, r, m_first);
     pdl_wait();
     cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
-    const int r = blockIdx.y;
     if (row_pos && row_pos[r] < 0) return;                       // the whole cluster leaves
     // first cluster barrier, split: arrive now, wait before the first access to another block's
     // shared memory (which is only legal once that block runs)
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     float ss = 0.f;
-    for (int m = m0 + threadIdx.x * 4; m < m1; m += blockDim.x * 4) {
-        float4 v = row_source_load4(src, r, m);
+    for (int m = m_first; m < m1; m += blockDim.x * 4) {
+        float4 v = (m == m_first && first_slots.n <= NQ) ? row_source_fetch<NQ>(first_slots) : row_source_load4(src, r, m);
         if (resid) {
             const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
@@ -369,15 +375,28 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
                                const int* __restrict__ row_seq, const float* __restrict__ cos_t,
                                const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
                                T* __restrict__ Kc, T* __restrict__ Vc, size_t seq_stride, size_t head_stride) {
-    pdl_enter();
+    pdl_trigger();
     const int r = blockIdx.x;
     const int half = head_dim / 2;
     T* qdst = q_t + (size_t)r * hidden;
+    // where the first group's q, k and v sums sit: arithmetic only, done before the wait for the GEMM
+    constexpr int NQ = 4;
+    const int m_first = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+    RowSlots<NQ> sq, sk, sv;
+    sq.n = NQ + 1;
+    if (m_first < hidden) {
+        sq = row_source_locate<NQ>(src, r, m_first);
+        sk = row_source_locate<NQ>(src, r, hidden + m_first);
+        sv = row_source_locate<NQ>(src, r, 2 * hidden + m_first);
+    }
+    pdl_wait();
     // four features = two rotary pairs per thread and turn
-    for (int m = (blockIdx.y * blockDim.x + threadIdx.x) * 4; m < hidden; m += gridDim.y * blockDim.x * 4) {
+    for (int m = m_first; m < hidden; m += gridDim.y * blockDim.x * 4) {
         // the sums are requested first; the row's position (and with it the rotary angles) meanwhile
-        const float4 q = row_source_load4(src, r, m), k = row_source_load4(src, r, hidden + m),
-                     v = row_source_load4(src, r, 2 * hidden + m);
+        const bool located = m == m_first && sq.n <= NQ && sk.n <= NQ && sv.n <= NQ;
+        const float4 q = located ? row_source_fetch<NQ>(sq) : row_source_load4(src, r, m),
+                     k = located ? row_source_fetch<NQ>(sk) : row_source_load4(src, r, hidden + m),
+                     v = located ? row_source_fetch<NQ>(sv) : row_source_load4(src, r, 2 * hidden + m);
         const int p = row_pos[r];
         if (p < 0) return;
         // cache layout [sequence][head][position][head_dim]: a head's keys are one contiguous stream
@@ -474,12 +493,19 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
 template <typename T>
 __global__ void swiglu_kernel(const RowSource src, int inner, T* __restrict__ act, size_t lda, int n_rows,
                               const int* __restrict__ row_pos) {
-    pdl_enter();
+    pdl_trigger();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t quads = (size_t)inner / 4;
-    if (i >= (size_t)n_rows * quads) return;
-    const int r = (int)(i / quads), j = (int)(i % quads) * 4;
-    const float4 g = row_source_load4(src, r, j), u = row_source_load4(src, r, inner + j);
+    const bool mine = i < (size_t)n_rows * quads;
+    const int r = mine ? (int)(i / quads) : 0, j = mine ? (int)(i % quads) * 4 : 0;
+    // where the gate and up sums sit: arithmetic only, done before the wait for the GEMM
+    constexpr int NQ = 4;
+    const RowSlots<NQ> sg = row_source_locate<NQ>(src, r, j), su = row_source_locate<NQ>(src, r, inner + j);
+    pdl_wait();
+    if (!mine) return;
+    const bool located = sg.n <= NQ && su.n <= NQ;
+    const float4 g = located ? row_source_fetch<NQ>(sg) : row_source_load4(src, r, j),
+                 u = located ? row_source_fetch<NQ>(su) : row_source_load4(src, r, inner + j);
     if (row_pos[r] < 0) return;
     const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll

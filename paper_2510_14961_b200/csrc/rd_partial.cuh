@@ -56,6 +56,55 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     }
     return acc;
 }
+// The same in two halves, for kernels that can do the index arithmetic before they wait for the GEMM:
+// where the (up to MAXQ) slots of features m..m+3 of row r are, then the loads and the ordered sum.
+template <int MAXQ>
+struct RowSlots {
+    const float* p[MAXQ];
+    int n;                // slots to add; n > MAXQ: not covered, use row_source_load4
+};
+template <int MAXQ>
+__device__ __forceinline__ RowSlots<MAXQ> row_source_locate(const RowSource& s, int r, int m) {
+    RowSlots<MAXQ> o;
+    if (s.plain) {
+        o.n = 1;
+        o.p[0] = s.plain + (size_t)r * s.ld + m;
+#pragma unroll
+        for (int q = 1; q < MAXQ; q++) o.p[q] = o.p[0];
+        return o;
+    }
+    const PartialSums& d = s.part;
+    const unsigned ft = (unsigned)(m >> 7);
+    const unsigned tile = (ft >> d.mt_shift) * d.n_tiles_n + (unsigned)(r / d.bn);
+    const unsigned t_lo = tile * (unsigned)d.kb;
+    const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
+    const size_t in_slot = ((size_t)(ft & ((1u << d.mt_shift) - 1)) * d.bn + (size_t)(r % d.bn)) * 128 + (m & 127);
+    const float* base = d.scratch + in_slot;
+    const size_t slot_elems = ((size_t)d.bn * 128) << d.mt_shift;
+    o.n = g_hi - g_lo + 1;
+#pragma unroll
+    for (int q = 0; q < MAXQ; q++) {
+        const unsigned g = (unsigned)(g_lo + min(q, g_hi - g_lo));
+        const unsigned first_tile = (g * (unsigned)d.per) / (unsigned)d.kb;
+        o.p[q] = base + ((size_t)g * d.max_seg + (tile - first_tile)) * slot_elems;
+    }
+    return o;
+}
+template <int MAXQ>
+__device__ __forceinline__ float4 row_source_fetch(const RowSlots<MAXQ>& o) {
+    float4 v[MAXQ];
+#pragma unroll
+    for (int q = 0; q < MAXQ; q++) {
+        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (q < o.n) v[q] = __ldcg(reinterpret_cast<const float4*>(o.p[q]));
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < MAXQ; q++)
+        if (q < o.n) { acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w; }
+    return acc;
+}
+
 __device__ __forceinline__ float row_source_load(const RowSource& s, int r, int m) {
     if (s.plain) return s.plain[(size_t)r * s.ld + m];
     const float4 v = row_source_load4(s, r, m & ~3);
