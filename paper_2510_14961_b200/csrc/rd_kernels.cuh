@@ -223,7 +223,7 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     }
     const int r = blockIdx.y;
     // where this thread's first group of four sits in the GEMM's scratch: arithmetic only, also before the wait
-    constexpr int NQ = 4;
+    constexpr int NQ = 8;      // out- and down-projection tiles are cut into up to 8 segments at 32 rows
     const int m_first = m0 + threadIdx.x * 4;
     RowSlots<NQ> first_slots;
     first_slots.n = NQ + 1;
@@ -499,7 +499,7 @@ __global__ void swiglu_kernel(const RowSource src, int inner, T* __restrict__ ac
     const bool mine = i < (size_t)n_rows * quads;
     const int r = mine ? (int)(i / quads) : 0, j = mine ? (int)(i % quads) * 4 : 0;
     // where the gate and up sums sit: arithmetic only, done before the wait for the GEMM
-    constexpr int NQ = 4;
+    constexpr int NQ = 2;      // a gate/up tile is cut into at most 2 segments at the model shapes here
     const RowSlots<NQ> sg = row_source_locate<NQ>(src, r, j), su = row_source_locate<NQ>(src, r, inner + j);
     pdl_wait();
     if (!mine) return;
