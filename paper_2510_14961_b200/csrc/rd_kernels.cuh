@@ -272,14 +272,18 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
 __global__ void reduce_store_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
                                     float* __restrict__ out, size_t ldo, int n, int n_rows,
                                     const int* __restrict__ row_pos, const int* __restrict__ row_steps, float eta) {
-    pdl_enter();
+    pdl_trigger();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if ((n & 3) == 0) {
         const size_t quads = (size_t)n / 4;
-        if (i >= (size_t)n_rows * quads) return;
-        const int r = (int)(i / quads), m = (int)(i % quads) * 4;
-        if (row_pos[r] < 0) return;
-        float4 v = row_source_load4(src, r, m);
+        const bool mine = i < (size_t)n_rows * quads;
+        const int r = mine ? (int)(i / quads) : 0, m = mine ? (int)(i % quads) * 4 : 0;
+        // slots located before the wait for the GEMM (arithmetic only)
+        constexpr int NQ = 8;
+        const RowSlots<NQ> sl = row_source_locate<NQ>(src, r, m);
+        pdl_wait();
+        if (!mine || row_pos[r] < 0) return;
+        float4 v = sl.n <= NQ ? row_source_fetch<NQ>(sl) : row_source_load4(src, r, m);
         if (resid) {
             const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
@@ -295,6 +299,7 @@ __global__ void reduce_store_kernel(const RowSource src, const float* __restrict
         }
         *dst = v;
     } else {
+        pdl_wait();
         const size_t per_row = ((size_t)n + 3) / 4;
         if (i >= (size_t)n_rows * per_row) return;
         const int r = (int)(i / per_row), m0 = (int)(i % per_row) * 4;
@@ -526,11 +531,18 @@ sample_scan_kernel(const RowSource src, int vocab, int chunk, const int* __restr
                    float* __restrict__ logits_store, float* __restrict__ best_val, int* __restrict__ best_idx) {
     __shared__ float sv[8];
     __shared__ int si[8];
-    pdl_enter();
+    pdl_trigger();
     const int r = blockIdx.x, ck = blockIdx.y;
+    const int v0 = ck * chunk, v1 = min(vocab, v0 + chunk);
+    // slots of this thread's first four logits, located before the wait for the head GEMM
+    constexpr int NQ = 4;
+    const int v_first = v0 + threadIdx.x * 4;
+    RowSlots<NQ> first_slots;
+    first_slots.n = NQ + 1;
+    if (v_first + 3 < vocab && (vocab & 3) == 0 && v_first < v1) first_slots = row_source_locate<NQ>(src, r, v_first);
+    pdl_wait();
     const int p = row_pos[r];
     if (p < 0) return;
-    const int v0 = ck * chunk, v1 = min(vocab, v0 + chunk);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     const uint32_t seq = (uint32_t)row_seq[r];
     float best = -INFINITY;
@@ -538,7 +550,7 @@ sample_scan_kernel(const RowSource src, int vocab, int chunk, const int* __restr
     for (int v = v0 + threadIdx.x * 4; v < v1; v += blockDim.x * 4) {
         float x[4];
         if (v + 3 < vocab && (vocab & 3) == 0) {
-            const float4 q = row_source_load4(src, r, v);
+            const float4 q = (v == v_first && first_slots.n <= NQ) ? row_source_fetch<NQ>(first_slots) : row_source_load4(src, r, v);
             x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
         } else {
 #pragma unroll
