@@ -63,11 +63,6 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "3p5b_b1_p512_g256_W32"
 
-# DRAM bytes (read + write) of one average GEMM launch of a step, from the ncu capture of the 32-row
-# GEMM summarised under profiles/ (taken on the 1/1/1-layer case with the same GEMM shapes; the head's
-# traffic scaled by vocabulary).  Valid for the kernel as profiled; set to None
-# when the GEMM kernel changes until the counters are taken again.
-NCU_GEMM_TRAFFIC_PER_LAUNCH = {"3p5b_b1_p512_g256_W32": 218.0e6}
 
 
 def max_over_ranks_sum_tokens(total_ms, tokens, dist=None, device=None):
@@ -83,6 +78,66 @@ def max_over_ranks_sum_tokens(total_ms, tokens, dist=None, device=None):
     return float(tm.item()), float(tk.item())
 
 
+def full_window_steps(gen, window):
+    """Fixed exit (Algorithm 1): rows are appended one per step, so after `window - 1` ramp steps the
+    wavefront holds `window` rows and every step commits one token per sequence, until the last of the
+    `gen` positions has been appended: steps window .. gen of a generation.  Returns that count."""
+    return max(0, gen - window + 1)
+
+
+def plan_timed_region(steps, gen, window):
+    """Segments (ramp_steps, timed_steps) that time exactly `steps` sampler steps at a full window.
+    Each segment restarts the generation (prefill, outside the timed region), runs `window - 1`
+    untimed ramp steps and then times up to full_window_steps(gen, window) steps.  A generation
+    shorter than its window never fills it: then the whole generation is the steady state there is,
+    and the segment times it from its first step (ramp 0)."""
+    if steps <= 0:
+        return []
+    full = full_window_steps(gen, window)
+    ramp = window - 1
+    if full <= 0:
+        ramp, full = 0, gen + window - 1
+    segs, left = [], steps
+    while left > 0:
+        n = min(left, full)
+        segs.append((ramp, n))
+        left -= n
+    return segs
+
+
+def expected_fixed_exit_tokens(segments, batch, gen, window):
+    """Tokens the fixed-exit sampler commits inside the timed segments: one per sequence and step at a
+    full window; for a generation that never fills its window, step t commits once t >= window."""
+    full = full_window_steps(gen, window)
+    tok = 0
+    for ramp, n in segments:
+        if full > 0:
+            tok += n * batch
+        else:
+            tok += batch * max(0, min(n, gen + window - 1) - (window - 1))
+    return tok
+
+
+def ncu_traffic_per_launch(workload):
+    """DRAM bytes (read + write) of one average GEMM launch from the ncu capture summarised in
+    profiles/, or None when the GEMM source has changed since the capture (the summary records the
+    sha256 of the kernel file it was taken with)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "gemm_tc_kernel_bn32_3p5b_shapes_W32.md")
+    src = os.path.join(ROOT, "paper_2510_14961_b200", "csrc", "rd_gemm_tc.cuh")
+    if workload != DEFAULT_WORKLOAD or not (os.path.exists(path) and os.path.exists(src)):
+        return None
+    traffic = sha = None
+    for line in open(path):
+        if line.startswith("traffic_bytes_per_launch:"):
+            traffic = float(line.split(":", 1)[1])
+        if line.startswith("kernel_source_sha256:"):
+            sha = line.split(":", 1)[1].strip()
+    if traffic is None or sha is None:
+        return None
+    return traffic if hashlib.sha256(open(src, "rb").read()).hexdigest() == sha else None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -90,6 +145,22 @@ def load_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
                     bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def prefill_flops(shape, lens, r):
+    """FLOPs of prefilling prompts of the given lengths (Section 3.3): rows 0..L-2 of each prompt go
+    through the prelude, r simultaneous core passes (adapter included) and the coda layers; causal
+    attention of row p costs 4 h (p + 1) per layer (QK^T and PV)."""
+    h, I = shape["hidden"], shape["mlp_inner"]
+    per_layer = 4 * h * h + 3 * h * I
+    n_p, n_r, n_c = shape["n_prelude"], shape["n_core"], shape["n_coda"]
+    w_elems = (n_p + n_c) * per_layer + r * (n_r * per_layer + 2 * h * h)
+    layers = n_p + n_c + r * n_r
+    total = 0
+    for L in lens:
+        n = max(int(L) - 1, 0)
+        total += 2 * n * w_elems + 4 * h * layers * (n * (n + 1) // 2)
+    return total
 
 
 def step_bytes_flops(shape, batch, rows, ctx_sum, inner, esz):
@@ -230,48 +301,90 @@ def run_ours(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     prefill(sess)                            # first call: also loads the kernels
     sess.sync()
-    t_pf0 = time.perf_counter()
+    ev0.record(stream)
     prefill(sess)
+    ev1.record(stream)
     sess.sync()
-    prefill_s = time.perf_counter() - t_pf0
-    for _ in range(max(args.warmup, 3)):
+    prefill_s = ev0.elapsed_time(ev1) * 1e-3
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
         sess.df_step(W, wl["inner"], wl["eps"])
     sess.sync()
-    if wl["eps"] <= 0:
+    adaptive = wl["eps"] > 0
+    if not adaptive:
         steps_per_gen = N + W - 1            # fixed exit: one token per step after the ramp
+        K = args.steps if args.steps > 0 else (full_window_steps(N, W) or steps_per_gen)
+        segments = plan_timed_region(K, N, W)
     else:
         # adaptive exit: the number of steps depends on the latents; an untimed generation with the
-        # same seeds counts them (every run of the same inputs takes the same steps)
+        # same seeds counts them (every run of the same inputs takes the same steps).  The timed
+        # region starts once the oldest row can have reached the iteration cap.
         prefill(sess)
         steps_per_gen = 0
         while not all(sess.committed(b)[1] for b in range(B)) and steps_per_gen < 64 * (N + W):
             sess.df_step(W, wl["inner"], wl["eps"])
             steps_per_gen += 1
-    K = args.steps if args.steps > 0 else steps_per_gen
+        if args.steps > 0:
+            ramp = min(max(W, -(-64 // wl["inner"])) - 1, max(steps_per_gen - 1, 0))
+            K = min(args.steps, steps_per_gen - ramp)
+            segments = [(ramp, K)]
+        else:
+            K = steps_per_gen
+            segments = [(0, K)]
+
+    def run_segments(segs):
+        """Times the segments' steps; returns (ms, tokens committed inside, kernel launches inside)."""
+        ms, tok, launches = 0.0, 0, 0
+        for ramp, n in segs:
+            prefill(sess)                   # restart the generation (outside the timed region)
+            for _ in range(ramp):
+                sess.df_step(W, wl["inner"], wl["eps"])
+            st0 = sess.stats()
+            barrier()
+            with torch.cuda.stream(stream):
+                ev0.record(stream)
+                for _ in range(n):
+                    sess.df_step(W, wl["inner"], wl["eps"])
+                ev1.record(stream)
+            barrier()
+            ms += ev0.elapsed_time(ev1)
+            st1 = sess.stats()
+            tok += st1["tokens_committed"] - st0["tokens_committed"]
+            launches += st1["kernel_launches"] - st0["kernel_launches"]
+        return ms, tok, launches
+
     clocks = ClockSampler(local)
     clocks.start()
-    total_ms, steps_done, tokens = 0.0, 0, 0
-    launches0 = None
-    while steps_done < K:
-        prefill(sess)                       # restart the generation (outside the timed region)
-        st0 = sess.stats()
-        n = min(K - steps_done, steps_per_gen)
-        barrier()
-        with torch.cuda.stream(stream):
-            ev0.record(stream)
-            for _ in range(n):
-                sess.df_step(W, wl["inner"], wl["eps"])
-            ev1.record(stream)
-        barrier()
-        total_ms += ev0.elapsed_time(ev1)
-        st1 = sess.stats()
-        tokens += st1["tokens_committed"] - st0["tokens_committed"]
-        launches0 = (launches0 or 0) + st1["kernel_launches"] - st0["kernel_launches"]
-        steps_done += n
+    reps = []
+    for _ in range(max(args.repeats, 1)):
+        ms, tok, launches0 = run_segments(segments)
+        ms_max, tok_all = max_over_ranks_sum_tokens(ms, tok, dist if world > 1 else None, dev)
+        reps.append((ms_max, tok_all))
     clk = clocks.stop()
-    total_ms_max, tokens_all = max_over_ranks_sum_tokens(total_ms, tokens, dist if world > 1 else None, dev)
+    if not adaptive:
+        want = expected_fixed_exit_tokens(segments, B, N, W)
+        if any(t != world * want for _, t in reps):
+            raise RuntimeError(f"timed region committed {[t for _, t in reps]} tokens, expected {world * want} per repeat")
+    rates = sorted(t / (m / 1e3) for m, t in reps)
+    if rates[len(rates) // 2] <= 0.0:
+        raise RuntimeError("the timed region committed no token: time more steps (adaptive exit commits in bursts)")
+    order = sorted(range(len(reps)), key=lambda i: reps[i][1] / reps[i][0])
+    total_ms_max, tokens_all = reps[order[len(order) // 2]]          # the median repeat
     df_tok_s = tokens_all / (total_ms_max / 1e3)
     ms_per_step = total_ms_max / K
+    timed_ctx_sum = sum(lens) + B * (sum(r + n / 2.0 for r, n in segments) / max(len(segments), 1))
+
+    # whole generation (ramp and drain included), timed once
+    prefill(sess)
+    barrier()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(steps_per_gen):
+            sess.df_step(W, wl["inner"], wl["eps"])
+        ev1.record(stream)
+    barrier()
+    gen_ms, gen_tok = max_over_ranks_sum_tokens(ev0.elapsed_time(ev1), B * N, dist if world > 1 else None, dev)
+    whole_generation_tok_s = gen_tok / (gen_ms / 1e3)
 
     # ---- per-kernel roofline: event pairs around every GEMM / attention launch -----------------
     prefill(sess)
@@ -287,12 +400,13 @@ def run_ours(args):
     gemm_gbs = prof["gemm_weight_bytes"] / (prof["gemm_ms"] * 1e-3) / 1e9 if prof["gemm_ms"] > 0 else 0.0
     attn_gbs = prof["attn_kv_bytes"] / (prof["attn_ms"] * 1e-3) / 1e9 if prof["attn_ms"] > 0 else 0.0
     tc_launches = sess.stats()["tc_gemm_launches"]
+    # step roofline for the steps that were timed: a full window of rows, the contexts they had
     rows_ss = B * W
-    ctx_mid = sum(lens) + B * (N // 2)
-    step_b, step_f = step_bytes_flops(shape, B, rows_ss, ctx_mid, wl["inner"], esz)
+    step_b, step_f = step_bytes_flops(shape, B, rows_ss, timed_ctx_sum, wl["inner"], esz)
     t_roof = max(step_b / (peaks["hbm_gbs"] * 1e9), step_f / (peaks["bf16_tflops_sustained"] * 1e12))
-    # steady-state step time: the steps profiled above ran with the full window
+    lib_stats = sess.stats()
     sess.close()
+    pf_flops = prefill_flops(shape, lens, wl["prefill_r"])
 
     # ---- AR decoder from the same library -------------------------------------------------------
     ar = new_session(1)
@@ -350,8 +464,13 @@ def run_ours(args):
 
     line = {
         "metric": "generated tok/s at 1 B200, DF sampler vs AR recurrence; % of step roofline",
-        "value": df_tok_s, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "value": df_tok_s, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": warm,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "repeats": {"n": len(reps), "statistic": "median", "tok_s": rates, "min": rates[0], "max": rates[-1]},
+        "timed_region": {"segments": [{"untimed_ramp_steps": r, "timed_steps": n} for r, n in segments],
+                         "what": "steps at a full window, every one committing" if not adaptive else
+                                 "steps after the ramp to the iteration cap (adaptive exit commits in bursts)"},
+        "whole_generation_tok_s": whole_generation_tok_s,
         "dtype": "bf16" if wl["bf16"] else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "prompt": L if len(set(lens)) == 1 else lens, "generate": N, "window": W,
                    "steps_per_generation": steps_per_gen, "tokens_per_step": tokens_all / (world * K) if K else None,
@@ -361,7 +480,9 @@ def run_ours(args):
                    "multi_gpu": "replicas only (no data-path collective)"},
         "df_tok_s": df_tok_s, "ar_tok_s": ar_tok_s, "df_over_ar": df_tok_s / ar_tok_s if ar_tok_s else None,
         "ar_tokens_timed": n_ar, "ar_ms_per_token": ar_ms / n_ar,
-        "prefill_s": prefill_s,
+        "prefill": {"seconds": prefill_s, "flops": pf_flops, "tflops": pf_flops / prefill_s / 1e12,
+                    "frac_of_bf16_sustained": pf_flops / prefill_s / 1e12 / peaks["bf16_tflops_sustained"],
+                    "prompts": L if len(set(lens)) == 1 else lens, "r": wl["prefill_r"], "timing": "CUDA events on the session's stream"},
         "step_roofline": {"bound": "hbm" if step_b / (peaks["hbm_gbs"] * 1e9) >= step_f / (peaks["bf16_tflops_sustained"] * 1e12) else "tensor",
                           "bytes_per_step": step_b, "flops_per_step": step_f, "t_roof_ms": t_roof * 1e3,
                           "df_frac": t_roof * 1e3 / ms_per_step,
@@ -369,7 +490,7 @@ def run_ours(args):
                           "peak_source": peaks["source"]},
         "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections of the step)",
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": NCU_GEMM_TRAFFIC_PER_LAUNCH.get(args.workload),
+                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(args.workload),
                      "launches": prof["gemm_launches"], "avg_us": 1e3 * prof["gemm_ms"] / max(prof["gemm_launches"], 1),
                      "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
                      "peak_source": peaks["source"]},
@@ -383,6 +504,7 @@ def run_ours(args):
                 "d2h_bytes_per_step": d2h / n_steps_e2e, "steps": n_steps_e2e, "prefill_s": e2e_prefill_s,
                 "total_s": e2e_s, "includes": "prompt upload, prefill, decode, per-step commit readback, token readback"},
         "gpu_launches": int(launches0), "tc_gemm_launches": int(tc_launches),
+        "library_counters": {k: lib_stats[k] for k in ("weight_bytes", "kv_bytes", "flops", "commit_hist") if k in lib_stats},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
@@ -489,8 +611,10 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=0, help="timed DF steps (default: one whole generation)")
+    ap.add_argument("--steps", type=int, default=0,
+                    help="timed DF steps at a full window (default: every full-window step of one generation)")
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--repeats", type=int, default=5, help="repeats of the timed region; the median is reported")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--ar-tokens", type=int, default=24)

@@ -94,6 +94,18 @@ typedef struct {
     uint64_t tokens_committed;             /* over all sequences, decode only                */
     uint64_t kernel_launches;              /* kernels of this library launched so far        */
     uint64_t tc_gemm_launches;             /* of those, tcgen05 GEMM launches                */
+    /* Algorithmic work of the decode steps enqueued so far (what the method must move and compute,
+     * cost remark of Section 3.5; not a measurement):                                         */
+    uint64_t weight_bytes;                 /* every weight matrix once per pass: prelude, coda and
+                                              head once per step, core and adapter once per inner
+                                              iteration                                        */
+    uint64_t kv_bytes;                     /* K and V: a sequence's cache rows 0..newest in-flight
+                                              position read once per layer and pass for its whole
+                                              window, plus the in-flight rows written          */
+    uint64_t flops;                        /* 2 per weight element and row, plus 4 * hidden per
+                                              (row, attended key, layer)                       */
+    uint64_t commit_hist[16];              /* (step, live sequence) pairs by tokens committed in
+                                              that step: [k] for k < 15, [15] for 15 or more   */
 } rd_stats_t;
 
 /* rd_load -- upload (or reference-free copy) of the weights of P, R, C (Section 3.1).
@@ -115,7 +127,11 @@ void rd_free(rd_model* m);
 /* rd_session_create -- allocate KV caches (three blocks, [layer][sequence][head][position][head_dim]),
  * latent slots and token arrays for `batch` sequences.
  *   cuda_stream   a cudaStream_t (as void*) on which every step is enqueued; NULL = legacy
- *                 default stream.  The model must outlive the session. */
+ *                 default stream.  The model must outlive the session.
+ * The model's device must be the current device (STATE otherwise); the first session on a device
+ * also sets that device's kernel attributes.  max_window may be at most 128 for RD_BF16 models whose
+ * head_dim is 64, 96 or 128 to stay on the tensor-core attention kernel (wider windows, other head
+ * sizes and RD_F32 run the one-row-per-block kernel).  batch * max_window <= 4096 (CAPACITY). */
 int rd_session_create(const rd_model* m, const rd_session_config* sc, void* cuda_stream,
                       rd_session** out);
 void rd_session_destroy(rd_session* s);
@@ -123,9 +139,11 @@ void rd_session_destroy(rd_session* s);
 /* rd_prefill -- Section 3.3: positions 0..n_prompt-2 of sequence `seq` run P, `r` simultaneous
  * passes of R (pass i of position p attends pass-i K/V of positions <= p) and the coda layers;
  * position n_prompt-1 becomes the first in-flight position with a fresh state (the initialisation
- * steps of Algorithm 1).  prompt: host pointer to n_prompt token ids in [0, vocab).  Re-prefilling a
- * sequence restarts it.  Errors: INVALID_ARG, CAPACITY (n_prompt + max_new_tokens >
- * max_context), OOM, CUDA. */
+ * steps of Algorithm 1).  prompt: host pointer to n_prompt token ids in [0, vocab); it is copied
+ * before the call returns.  The call only ENQUEUES the work on the session's stream (upload of the
+ * prompt, the passes, the sequence's new state) and returns; it allocates nothing.  Re-prefilling a
+ * sequence restarts it; the other sequences of the session keep their wavefronts and go on with the
+ * next step.  Errors: INVALID_ARG, CAPACITY (n_prompt + max_new_tokens > max_context), CUDA. */
 int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r);
 
 /* rd_ar_step -- one token on every live sequence by the sequential recurrence (Section 3.1):
@@ -199,6 +217,17 @@ int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int32_t which,
  *     the same device (two host threads, two sessions) race on it: serialise them. */
 int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t layer, int32_t which, int32_t seq,
                              int32_t pos0, int32_t n, float* dst);
+
+/* rd_debug_expire_next_wait -- test aid for the RD_E_TIMEOUT path.  Every wait of a GEMM kernel on a
+ * pipeline barrier is bounded; when one runs out the kernel raises the session's status word, lets
+ * the copies it issued land, frees its tensor memory and returns, and rd_sync reports RD_E_TIMEOUT
+ * from then on (the session can still be destroyed, and other sessions are unaffected).  This call
+ * makes that happen once: in the next tensor-core GEMM launch on single CTAs, one CTA never requests
+ * the first operand tile of its share, so the barrier that tile would complete stays incomplete, and
+ * the launch's waits give up after a few thousand polls instead of millions.  Nothing faults and no
+ * wait is unbounded; the step's results are meaningless.  STATE when the session has no tensor-core
+ * GEMM path. */
+int rd_debug_expire_next_wait(rd_session* s);
 
 /* rd_stats -- counters since session creation (host pointer out). */
 int rd_stats(rd_session* s, rd_stats_t* out);

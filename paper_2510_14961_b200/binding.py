@@ -17,7 +17,8 @@ RD_DBG_LATENTS, RD_DBG_DELTA, RD_DBG_DRAFTS, RD_DBG_LOGITS, RD_DBG_EMBED = 0, 1,
 EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_prefill", "rd_ar_step",
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
-           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining"]
+           "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining",
+           "rd_debug_expire_next_wait"]
 
 
 class RdConfig(C.Structure):
@@ -35,7 +36,8 @@ class RdSessionConfig(C.Structure):
 
 class RdStats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("df_steps", "ar_steps", "rows_prelude", "rows_core", "rows_coda",
-                                          "tokens_committed", "kernel_launches", "tc_gemm_launches")]
+                                          "tokens_committed", "kernel_launches", "tc_gemm_launches",
+                                          "weight_bytes", "kv_bytes", "flops")] + [("commit_hist", C.c_uint64 * 16)]
 
 
 class RdProfile(C.Structure):
@@ -81,6 +83,7 @@ def lib():
         L.rd_stats.argtypes = [vp, C.POINTER(RdStats)]
         L.rd_set_gemm_path.argtypes = [vp, i32]
         L.rd_set_launch_chaining.argtypes = [vp, i32]
+        L.rd_debug_expire_next_wait.argtypes = [vp]
         L.rd_profile_enable.argtypes = [vp, i32]
         L.rd_profile_read.argtypes = [vp, C.POINTER(RdProfile)]
         L.rd_strerror.argtypes = [C.c_int]
@@ -223,13 +226,19 @@ class Session:
     def stats(self):
         st = RdStats()
         _check(lib().rd_stats(self.handle, C.byref(st)), "rd_stats")
-        return {k: getattr(st, k) for k, _ in RdStats._fields_}
+        out = {k: getattr(st, k) for k, _ in RdStats._fields_}
+        out["commit_hist"] = [int(v) for v in st.commit_hist]
+        return out
 
     def set_gemm_path(self, path):
         _check(lib().rd_set_gemm_path(self.handle, path), "rd_set_gemm_path")
 
     def set_launch_chaining(self, on):
         _check(lib().rd_set_launch_chaining(self.handle, 1 if on else 0), "rd_set_launch_chaining")
+
+    def expire_next_wait(self):
+        """Test aid: the next tensor-core GEMM launch lets one bounded wait run out (RD_E_TIMEOUT at the next sync)."""
+        _check(lib().rd_debug_expire_next_wait(self.handle), "rd_debug_expire_next_wait")
 
     def profile_enable(self, on=True):
         _check(lib().rd_profile_enable(self.handle, 1 if on else 0), "rd_profile_enable")

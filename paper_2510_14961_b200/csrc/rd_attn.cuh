@@ -1,8 +1,8 @@
 // Windowed flash-decode attention for the bf16 path.
 //
-// One CTA takes one (query group, head, KV split).  A query group is a set of up to 64 rows of ONE
-// sequence (the in-flight wavefront of a sequence during decode, 64 consecutive prompt positions
-// during prefill).  The row at position p attends cache entries 0..p of its sequence: committed
+// One CTA takes one (query group, head, KV split).  A query group is a set of up to 128 rows of ONE
+// sequence (the in-flight wavefront of a sequence during decode, 128 consecutive prompt positions
+// during prefill); a CTA has one warp per 16 queries of the largest group it takes (4 or 8 warps).  The row at position p attends cache entries 0..p of its sequence: committed
 // prefix and the in-flight rows <= p as overwritten this pass (shared KV cache, Section 3.2;
 // causal, left to right only).  K and V tiles of 64 keys stream through shared memory once per CTA
 // (16-byte cp.async, double buffered) and are reused by every query of the group, so the KV
@@ -23,7 +23,7 @@
 namespace rd {
 
 constexpr int ATT_KT = 64;          // keys per tile
-constexpr int ATT_QMAX = 64;        // queries per group
+constexpr int ATT_QMAX = 128;       // queries per group (the paper's default maximum wavefront)
 constexpr int ATT_MAX_SPLITS = 8;    // = portable cluster size
 
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
@@ -54,14 +54,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-template <int D> struct AttCfg {
+template <int D, int NW> struct AttCfg {
     static constexpr int LD = D + 8;    // padded row (elements): ldmatrix rows fall in distinct banks
-    static constexpr int SMEM = (ATT_QMAX * LD + 4 * ATT_KT * LD) * 2 + ATT_QMAX * 4;
+    static constexpr int QMAX = 16 * NW;   // queries a CTA of NW warps holds
+    static constexpr int SMEM = (QMAX * LD + 4 * ATT_KT * LD) * 2 + QMAX * 4;
 };
 
 // Grid (splits, heads, groups), clusters of `splits` blocks along x.  out: [rows, hidden] bf16.
-// KW = keys of a 64-key tile one warp takes.  KW = 64: the four warps are four blocks of 16 queries
-// (groups of up to 64 rows).  KW = 32, for groups of at most 32 rows: warps 0,1 take the two query
+// KW = keys of a 64-key tile one warp takes.  KW = 64: the NW warps are NW blocks of 16 queries
+// (groups of up to 16 NW rows: 64 with four warps, 128 with eight).  KW = 32, for groups of at most 32 rows: warps 0,1 take the two query
 // blocks on the tile's first 32 keys, warps 2,3 the same queries on its last 32, and the two halves
 // are merged (first half, then second) through shared memory before the cluster merge.
 // Groups in the order the hardware should start them (blockIdx.z counts through it): the host
@@ -72,17 +73,20 @@ struct GroupOrder {
     int n;                              // 0: groups in index order
 };
 
-template <int D, int KW>
-__global__ void __launch_bounds__(128)
+template <int D, int KW, int NW>
+__global__ void __launch_bounds__(32 * NW)
 attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
                    const int* __restrict__ row_seq, int rows_per_group, int n_rows,
                    const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
                    size_t head_stride, int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
-    constexpr int LD = AttCfg<D>::LD;
+    constexpr int LD = AttCfg<D, NW>::LD;
+    constexpr int QMAX = AttCfg<D, NW>::QMAX;
+    constexpr int NT = 32 * NW;
     constexpr int CH = D / 8;           // 16-byte chunks per row
+    static_assert(KW == 64 || NW == 4, "half-tile warps only with four warps");
     extern __shared__ __align__(16) uint8_t att_smem[];
     __nv_bfloat16* Qs = (__nv_bfloat16*)att_smem;
-    __nv_bfloat16* Ks = Qs + ATT_QMAX * LD;               // [2][KT][LD]
+    __nv_bfloat16* Ks = Qs + QMAX * LD;                   // [2][KT][LD]
     __nv_bfloat16* Vs = Ks + 2 * ATT_KT * LD;             // [2][KT][LD]
     int* pos_s = (int*)(Vs + 2 * ATT_KT * LD);
 
@@ -92,13 +96,15 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     const int r0 = (order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z) * rows_per_group;
     const int nq = min(rows_per_group, n_rows - r0);
     // positions of the group's rows; kv_len = 1 + the largest of them
-    __shared__ int warp_max[4];
-    const int my_pos = (tid < ATT_QMAX && tid < nq) ? row_pos[r0 + tid] : -1;
-    if (tid < ATT_QMAX) pos_s[tid] = my_pos;
+    __shared__ int warp_max[NW];
+    const int my_pos = (tid < QMAX && tid < nq) ? row_pos[r0 + tid] : -1;
+    if (tid < QMAX) pos_s[tid] = my_pos;
     const int wmax = __reduce_max_sync(0xffffffffu, my_pos);
     if (lane == 0) warp_max[warp] = wmax;
     __syncthreads();
-    const int kv_len = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3])) + 1;
+    int kv_len = 0;
+#pragma unroll
+    for (int w = 0; w < NW; w++) kv_len = max(kv_len, warp_max[w] + 1);
     const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
     const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
     const int seq = row_seq[r0];
@@ -106,7 +112,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     const __nv_bfloat16* kbase = Kc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
     const __nv_bfloat16* vbase = Vc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
 
-    for (int c = tid; c < ATT_QMAX * CH; c += 128) {
+    for (int c = tid; c < QMAX * CH; c += NT) {
         const int r = c / CH, ch = c % CH;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)(r0 + r) * hidden + hd * D + ch * 8);
@@ -114,7 +120,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     }
     auto load_tile = [&](int t, int buf) {
         const int key0 = t * ATT_KT;
-        for (int c = tid; c < ATT_KT * CH; c += 128) {
+        for (int c = tid; c < ATT_KT * CH; c += NT) {
             const int r = c / CH, ch = c % CH;
             const int key = key0 + r;
             const bool ok = key < kv_len;
@@ -214,13 +220,13 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
         __syncthreads();                                   // buffer may be refilled next round
     }
     // ---- partials to shared memory (the K/V buffers are free now), merge across the cluster ----
-    float* Os = reinterpret_cast<float*>(att_smem);          // [ATT_QMAX][D] unnormalised outputs
-    float* MLs = Os + ATT_QMAX * D;                           // [ATT_QMAX][2] (max in the log2 domain, sum)
+    float* Os = reinterpret_cast<float*>(att_smem);          // [QMAX][D] unnormalised outputs
+    float* MLs = Os + QMAX * D;                               // [QMAX][2] (max in the log2 domain, sum)
     __syncthreads();
     if (KW != 64) {
         // the warps of the second key half hand (m, l, O) to the warps of the first half, thread to thread
         constexpr int PER = D / 2 + 4;
-        float* st = MLs + ATT_QMAX * 2 + (size_t)(qblk * 32 + lane) * PER;
+        float* st = MLs + QMAX * 2 + (size_t)(qblk * 32 + lane) * PER;
         if (warp >= 2) {
 #pragma unroll
             for (int j = 0; j < D / 8; j++)
@@ -271,7 +277,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     // block `sp` merges queries sp, sp + n_splits, ...; one thread per 4 output elements
     constexpr int Q4 = D / 4;
     const int mine = nq > sp ? (nq - sp + n_splits - 1) / n_splits : 0;
-    for (int item = tid; item < mine * Q4; item += 128) {
+    for (int item = tid; item < mine * Q4; item += NT) {
         const int q = sp + (item / Q4) * n_splits, e = (item % Q4) * 4;
         __nv_bfloat16* dst = out + (size_t)(r0 + q) * hidden + hd * D + e;
         float2 ml[ATT_MAX_SPLITS];

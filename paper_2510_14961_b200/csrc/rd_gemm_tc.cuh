@@ -140,9 +140,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < TC_SPIN_LIMIT; i++) {
+// Bounded wait: false when `limit` polls ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = TC_SPIN_LIMIT) {
+    for (uint32_t i = 0; i < limit; i++) {
         if (mbar_test(bar, parity)) return true;
         if (i > 64) __nanosleep(64);
     }
@@ -294,6 +294,10 @@ struct TcParams {
     int max_seg;               // scratch slots per CTA
     float* scratch;            // [gridDim.x * max_seg][MT][BN][128] partial sums
     int* status;
+    uint32_t spin_limit;       // polls a wait on a pipeline barrier may take (TC_SPIN_LIMIT)
+    int skip_unit;             // -1.  Test aid (rd_debug_expire_next_wait): CTA 0's producer leaves this unit of
+                               // its share out, so that the barrier the unit would complete is never completed
+                               // and the waits on it run out
 };
 
 template <int BN>
@@ -331,7 +335,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             // Weights do not depend on the previous kernel: the first ring of A tiles is requested
             // before the dependency wait, the matching B tiles after it.
             const int pre = min(n_units, C::STAGES);
+            const int skip = blockIdx.x == 0 ? p.skip_unit : -1;   // test aid: a unit among the first `pre` that is never loaded
             for (int i = 0; i < pre; i++) {
+                if (i == skip) continue;
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], C::STAGE_BYTES);
@@ -339,6 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
+                if (i == skip) continue;
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[i]);
@@ -346,7 +353,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             int issued = pre;
             for (int i = pre; i < n_units; i++) {
                 const int s = i % C::STAGES;
-                if (*abort_flag || !mbar_wait(&empty[s], ((i / C::STAGES) - 1) & 1)) { *abort_flag = 1; break; }
+                if (*abort_flag || !mbar_wait(&empty[s], ((i / C::STAGES) - 1) & 1, p.spin_limit)) { *abort_flag = 1; break; }
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[s], C::STAGE_BYTES);
@@ -357,7 +364,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             }
             if (*abort_flag) {
                 // drain: every stage this thread armed must land before the CTA's memory is released
-                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1);
+                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1, p.spin_limit);
             }
         } else {
             pdl_wait();
@@ -380,12 +387,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     const int ka = (int)(u % p.kb);
                     const int len = min(p.kb - ka, n_units - i);
                     const int buf = seg % C::NBUF, use = seg / C::NBUF;
-                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1)) { ok = false; break; }
+                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1, p.spin_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d = tmem_base + (uint32_t)(buf * C::MT * C::ACC_COLS);
                     for (int j = 0; j < len; j++, i++) {
                         const int s = i % C::STAGES;
-                        if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1)) { ok = false; break; }
+                        if (*abort_flag || !mbar_wait(&full[s], (i / C::STAGES) & 1, p.spin_limit)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t a = smem_u32(smem + s * C::STAGE_BYTES);
                         const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
@@ -413,7 +420,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int ka = (int)(u % p.kb);
                 const int len = min(p.kb - ka, n_units - i);
                 const int buf = seg % C::NBUF;
-                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1)) { ok = false; break; }
+                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1, p.spin_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::MT * C::ACC_COLS);
                 // the share's seg-th segment (= seg-th tile it touches) -> slot blockIdx.x * max_seg + seg
@@ -550,7 +557,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             int s = pre % C::STAGES;
             uint32_t parity = (uint32_t)(((pre / C::STAGES) - 1) & 1);
             for (int i = pre; i < n_units; i++) {
-                if (*abort_flag || !mbar_wait(&empty[s], parity)) { *abort_flag = 1; break; }
+                if (*abort_flag || !mbar_wait(&empty[s], parity, p.spin_limit)) { *abort_flag = 1; break; }
                 if (rank == 0) mbar_expect_tx(&full[s], 2 * C::STAGE_BYTES);
                 uint8_t* a = smem + s * C::STAGE_BYTES;
                 const uint32_t bar = map_to_rank(&full[s], 0);
@@ -562,7 +569,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
             }
             if (*abort_flag && rank == 0) {
                 // drain: the stages the leader armed count both CTAs' bytes
-                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1);
+                for (int i = max(0, issued - C::STAGES); i < issued; i++) mbar_wait(&full[i % C::STAGES], (i / C::STAGES) & 1, p.spin_limit);
             }
         } else {
             pdl_wait();
@@ -586,11 +593,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                     const int ka = (int)(u % p.kb);
                     const int len = min(p.kb - ka, n_units - i);
                     const int buf = seg % C::NBUF, use = seg / C::NBUF;
-                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1)) { ok = false; break; }
+                    if (use >= 1 && !mbar_wait(&acc_empty[buf], (use - 1) & 1, p.spin_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d = tmem_base + (uint32_t)(buf * C::ACC_COLS);
                     for (int j = 0; j < len; j++, i++) {
-                        if (*abort_flag || !mbar_wait(&full[s], parity)) { ok = false; break; }
+                        if (*abort_flag || !mbar_wait(&full[s], parity, p.spin_limit)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t a = smem_u32(smem + s * C::STAGE_BYTES);
                         const uint64_t adesc = umma_desc_k128(a), bdesc = umma_desc_k128(a + C::A_BYTES);
@@ -617,7 +624,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 const int ka = (int)(u % p.kb);
                 const int len = min(p.kb - ka, n_units - i);
                 const int buf = seg % C::NBUF;
-                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1)) { ok = false; break; }
+                if (*abort_flag || !mbar_wait(&acc_full[buf], (seg / C::NBUF) & 1, p.spin_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::ACC_COLS);
                 // slot of the pair's seg-th segment; this CTA's feature tile is the rank-th of the unit's two
@@ -688,39 +695,51 @@ static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair 
 
 template <int BN>
 static int tc_launch(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, int grid, bool chained) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM) != cudaSuccess)
-            return RD_E_CUDA;
-        attr_set = true;
-    }
     return launch_chained(gemm_tc_kernel<BN>, dim3(grid), dim3(TC_THREADS), TcCfg<BN>::SMEM, st, chained, mw, mx, p) == cudaSuccess
                ? RD_OK : RD_E_CUDA;
 }
 
 template <int BN>
 static int tc_launch_pair(cudaStream_t st, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, int pairs, bool chained) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcPairCfg<BN>::SMEM) != cudaSuccess)
-            return RD_E_CUDA;
-        attr_set = true;
-    }
     return launch_chained_cluster(gemm_tc_pair_kernel<BN>, dim3(2 * pairs), dim3(TC_THREADS), TcPairCfg<BN>::SMEM, st, chained, 2, mw, mx, p) ==
                    cudaSuccess ? RD_OK : RD_E_CUDA;
+}
+
+// Opt-in to more than 48 KB of dynamic shared memory for every GEMM kernel, on the CURRENT device
+// (the attribute is kept per device: call once for each device a session is created on).
+static inline int tc_configure_device() {
+    cudaError_t e = cudaSuccess;
+    auto set = [&](auto* kern, int smem) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    };
+    set(gemm_tc_kernel<16>, TcCfg<16>::SMEM);
+    set(gemm_tc_kernel<32>, TcCfg<32>::SMEM);
+    set(gemm_tc_kernel<64>, TcCfg<64>::SMEM);
+    set(gemm_tc_kernel<128>, TcCfg<128>::SMEM);
+    set(gemm_tc_kernel<256>, TcCfg<256>::SMEM);
+    set(gemm_tc_pair_kernel<128>, TcPairCfg<128>::SMEM);
+    set(gemm_tc_pair_kernel<256>, TcPairCfg<256>::SMEM);
+    return e == cudaSuccess ? RD_OK : RD_E_CUDA;
 }
 
 // Launches the GEMM; *out describes where a consumer finds the sums.  Returns RD_E_INVALID_ARG when
 // the shape is not taken (caller falls back to the SIMT kernels).
 static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
                           float* scratch, size_t scratch_elems, int n_sms, int* status, bool chained, PartialSums* out,
-                          bool pair = true) {
+                          bool pair = true, bool* expire_wait = nullptr) {
     if (ta.K != K || tw.K != K || tw.n_out != n_out || n_rows < 1 || n_rows > ta.rows) return RD_E_INVALID_ARG;
     const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms, pair);
     if (pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
     p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
     p.scratch = scratch; p.status = status;
+    p.spin_limit = TC_SPIN_LIMIT; p.skip_unit = -1;
+    if (expire_wait && *expire_wait && !pl.pair) {
+        // test aid, one launch: CTA 0 never loads the first unit of its share and every wait of the
+        // launch gives up after a few thousand polls; the kernel then raises the status word
+        p.spin_limit = 1u << 12; p.skip_unit = 0;
+        *expire_wait = false;
+    }
     out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_n = pl.n_tiles_n; out->bn = pl.bn;
     out->max_seg = pl.max_seg; out->mt_shift = pl.mt == 2 ? 1 : 0;
     switch (pl.bn_idx) {

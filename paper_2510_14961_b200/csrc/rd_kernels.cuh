@@ -905,10 +905,16 @@ delta_kernel(const float* __restrict__ z, const float* __restrict__ z_prev, int 
 struct SeqState {
     int* n_prompt; int* n_committed; int* win_len; int* done;
     int* row_steps; int* row_iters;
-    unsigned long long* counters;   // [0] rows through P, [1] R, [2] C, [3] tokens committed
+    unsigned long long* counters;   // [0] rows through P, [1] R, [2] C, [3] tokens committed,
+                                    // [4] cache rows read (context of a sequence, once per layer and pass),
+                                    // [5] (row, attended key) pairs summed over layers and passes,
+                                    // [8 + k] (step, live sequence) pairs that committed k tokens (k = 15: 15 or more)
 };
+constexpr int RD_COUNTERS = 32;
+constexpr int RD_HIST_AT = 8, RD_HIST_BINS = 16;
+// layer_passes: layers a row goes through in this step (prelude + coda + inner_iters * core).
 __global__ void advance_kernel(SeqState st, const float* __restrict__ delta, int B, int Wmax, int window,
-                               int inner_iters, float exit_threshold, int cap, int max_new) {
+                               int inner_iters, float exit_threshold, int cap, int max_new, int layer_passes) {
     pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B || st.done[b]) return;
@@ -926,12 +932,17 @@ __global__ void advance_kernel(SeqState st, const float* __restrict__ delta, int
     atomicAdd(&st.counters[0], (unsigned long long)w);
     atomicAdd(&st.counters[1], (unsigned long long)w * inner_iters);
     atomicAdd(&st.counters[2], (unsigned long long)w);
+    // rows at positions f .. f+w-1: the cache rows 0 .. f+w-1 are read once for the whole window;
+    // the row at position p attends p + 1 keys
+    atomicAdd(&st.counters[4], (unsigned long long)(f + w) * layer_passes);
+    atomicAdd(&st.counters[5], ((unsigned long long)w * (f + 1) + (unsigned long long)w * (w - 1) / 2) * layer_passes);
     int nc = st.n_committed[b];
     const int np = st.n_prompt[b];
     k = min(k, max_new - (nc - np));
     nc += k;
     w -= k;
     atomicAdd(&st.counters[3], (unsigned long long)k);
+    atomicAdd(&st.counters[RD_HIST_AT + min(k, RD_HIST_BINS - 1)], 1ull);
     if (nc - np >= max_new) {
         st.done[b] = 1;
         w = 0;
@@ -946,6 +957,19 @@ __global__ void advance_kernel(SeqState st, const float* __restrict__ delta, int
     }
     st.n_committed[b] = nc;
     st.win_len[b] = w;
+}
+
+// End of a prefill, on the stream: |y_frozen| = L and one fresh in-flight row at position L-1
+// (the initialisation steps of Algorithm 1).
+__global__ void seq_start_kernel(SeqState st, int seq, int L, int slot, int is_done) {
+    pdl_enter();
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    st.n_prompt[seq] = L;
+    st.n_committed[seq] = L;
+    st.win_len[seq] = is_done ? 0 : 1;
+    st.done[seq] = is_done;
+    st.row_steps[slot] = 0;
+    st.row_iters[slot] = 0;
 }
 
 // float32 -> T copy (weight upload path; bf16 rounds to nearest even once).

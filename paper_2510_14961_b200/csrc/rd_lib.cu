@@ -242,6 +242,12 @@ struct rd_session {
     size_t tc_scratch_elems = 0;
     float* best_val = nullptr;     // per (row, vocabulary chunk): best score and its index
     int* best_idx = nullptr;
+    float *pf_e = nullptr, *pf_s = nullptr;   // prefill workspace: e and the latent of every prompt row, [max_context, h]
+    static constexpr int PROMPT_STAGES = 4;   // pinned copies of the prompts being uploaded (the caller's buffer is only borrowed)
+    int* prompt_stage[PROMPT_STAGES] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t prompt_ev[PROMPT_STAGES] = {nullptr, nullptr, nullptr, nullptr};
+    int stage_next = 0;
+    bool expire_next_wait = false;            // test aid: see rd_debug_expire_next_wait
     float* acc = nullptr;          // output of the plain GEMM kernel, [rows, n_out]
     size_t acc_elems = 0;
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
@@ -266,6 +272,10 @@ struct rd_session {
     uint64_t ctx_total = 0;   // host-side upper bound of sum over sequences of context length
     ~rd_session() {
         if (mirror) cudaFreeHost(mirror);
+        for (int i = 0; i < PROMPT_STAGES; i++) {
+            if (prompt_stage[i]) cudaFreeHost(prompt_stage[i]);
+            if (prompt_ev[i]) cudaEventDestroy(prompt_ev[i]);
+        }
         for (Bracket& b : brackets) { cudaEventDestroy(b.a); cudaEventDestroy(b.b); }
         for (cudaEvent_t e : event_pool) cudaEventDestroy(e);
     }
@@ -309,10 +319,26 @@ template <typename T> static void want_max_carveout_typed() {
     want_max_carveout(attn_row_kernel<T>);
     want_max_carveout(swiglu_kernel<T>);
 }
-static void want_max_carveout_everywhere() {
-    static bool done = false;
-    if (done) return;
-    done = true;
+template <int D> static cudaError_t attn_configure_d() {
+    cudaError_t e = cudaSuccess;
+    auto set = [&](auto* kern, int smem) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        want_max_carveout(kern);
+    };
+    set(attn_window_kernel<D, 32, 4>, AttCfg<D, 4>::SMEM);
+    set(attn_window_kernel<D, 64, 4>, AttCfg<D, 4>::SMEM);
+    set(attn_window_kernel<D, 64, 8>, AttCfg<D, 8>::SMEM);
+    return e;
+}
+// Function attributes (shared-memory opt-in, carve-out preference) are kept per device: they are
+// set once for every device a session is created on, with that device current.
+constexpr int RD_MAX_DEVICES = 64;
+static bool g_device_configured[RD_MAX_DEVICES];
+static std::mutex g_device_mutex;
+static int configure_device_kernels(int device) {
+    if (device < 0 || device >= RD_MAX_DEVICES) return RD_E_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    if (g_device_configured[device]) return RD_OK;
     want_max_carveout_typed<float>();
     want_max_carveout_typed<bf16>();
     want_max_carveout(plan_rows_kernel);
@@ -323,7 +349,14 @@ static void want_max_carveout_everywhere() {
     want_max_carveout(sample_pick_kernel);
     want_max_carveout(delta_kernel);
     want_max_carveout(advance_kernel);
-    cudaGetLastError();   // an attribute a kernel does not take is not an error of the session
+    cudaGetLastError();   // a preference a kernel does not take is not an error of the session
+    if (tc_configure_device() != RD_OK) return cuda_fail(cudaGetLastError(), "shared-memory opt-in of the GEMM kernels", __LINE__);
+    cudaError_t e = attn_configure_d<64>();
+    if (e == cudaSuccess) e = attn_configure_d<96>();
+    if (e == cudaSuccess) e = attn_configure_d<128>();
+    if (e != cudaSuccess) return cuda_fail(e, "shared-memory opt-in of the attention kernels", __LINE__);
+    g_device_configured[device] = true;
+    return RD_OK;
 }
 
 extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp, void* cuda_stream,
@@ -337,9 +370,14 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     // the top-p kernel keeps a row's logits in the registers of one cluster
     if (sc.temperature > 0.f && sc.top_p > 0.f && sc.top_p < 1.f && m->cfg.vocab > NUC_MAX_VOCAB) return RD_E_INVALID_ARG;
     if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
+    {
+        int dev = -1;
+        CU(cudaGetDevice(&dev));
+        if (dev != m->device) return RD_E_STATE;      // the model's device must be current
+        RD_TRY(configure_device_kernels(dev));
+    }
     rd_session* s = new (std::nothrow) rd_session();
     if (!s) return RD_E_OOM;
-    want_max_carveout_everywhere();
     s->m = m;
     s->sc = sc;
     s->stream = (cudaStream_t)cuda_stream;
@@ -365,7 +403,7 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if ((rc = s->mem.get(&s->row_pos, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->row_seq, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->draft, R * sizeof(int)))) break;
-        if ((rc = s->mem.get(&s->counters, 8 * sizeof(unsigned long long)))) break;
+        if ((rc = s->mem.get(&s->counters, RD_COUNTERS * sizeof(unsigned long long)))) break;
         // what the host polls sits in one block (status word, |y_frozen| and done flag per sequence)
         // so that one copy into a pinned mirror brings all of it
         s->poll_ints = 4 + 2 * B;
@@ -376,6 +414,16 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
             cudaError_t eh = cudaHostAlloc((void**)&s->mirror, s->poll_ints * sizeof(int), cudaHostAllocDefault);
             if (eh != cudaSuccess) { rc = cuda_fail(eh, "cudaHostAlloc", __LINE__); break; }
         }
+        {
+            cudaError_t eh = cudaSuccess;
+            for (int i = 0; i < rd_session::PROMPT_STAGES && eh == cudaSuccess; i++) {
+                eh = cudaHostAlloc((void**)&s->prompt_stage[i], (size_t)s->tok_stride * sizeof(int), cudaHostAllocDefault);
+                if (eh == cudaSuccess) eh = cudaEventCreateWithFlags(&s->prompt_ev[i], cudaEventDisableTiming);
+            }
+            if (eh != cudaSuccess) { rc = cuda_fail(eh, "prompt staging", __LINE__); break; }
+        }
+        if ((rc = s->mem.get(&s->pf_e, (size_t)sc.max_context * h * sizeof(float)))) break;
+        if ((rc = s->mem.get(&s->pf_s, (size_t)sc.max_context * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->x, R * h * sizeof(float)))) break;
         s->acc_elems = std::max(R * std::max<size_t>(std::max<size_t>(3 * h, 2 * I), h), (size_t)s->n_slots * V);
         if ((rc = s->mem.get(&s->acc, s->acc_elems * sizeof(float)))) break;
@@ -514,7 +562,7 @@ template <typename T> struct Eng {
         *out = RowSource{};
         if (tc_usable(s, ta, tw)) {
             const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, n_rows, s->tc_scratch, s->tc_scratch_elems, s->m->n_sms,
-                                   s->status, s->chained, &out->part, s->gemm_path == 1);
+                                   s->status, s->chained, &out->part, s->gemm_path == 1, &s->expire_next_wait);
             if (rc == RD_OK) {
                 s->stats.tc_gemm_launches++; s->stats.kernel_launches++;
                 bracket_close(s, br);
@@ -553,14 +601,8 @@ template <typename T> struct Eng {
     }
 
     // Windowed flash-decode attention (bf16): groups of s->grp_rows rows share their sequence's KV.
-    template <int D, int KW>
+    template <int D, int KW, int NW>
     static int attn_windowed_d(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
-        static bool attr_set = false;
-        if (!attr_set) {
-            CU(cudaFuncSetAttribute(attn_window_kernel<D, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttCfg<D>::SMEM));
-            cudaFuncSetAttribute(attn_window_kernel<D, KW>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-            attr_set = true;
-        }
         const rd_config& c = s->m->cfg;
         const int groups = (n_rows + s->grp_rows - 1) / s->grp_rows;
         const int tiles = std::max(1, (s->ctx_max + ATT_KT - 1) / ATT_KT);
@@ -578,15 +620,18 @@ template <typename T> struct Eng {
             for (int g = 0; g < groups; g++) order.idx[g] = (unsigned char)ids[g];
             order.n = groups;
         }
-        LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW>), (ns, c.n_heads, groups), 128, AttCfg<D>::SMEM, ns, order, (const bf16*)s->q_t,
+        LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttCfg<D, NW>::SMEM), ns, order, (const bf16*)s->q_t,
                        s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
                        (bf16*)s->act_h);
         return RD_OK;
     }
     template <int D>
     static int attn_windowed_k(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
-        // groups of at most 32 rows: every warp takes half of a key tile, so all four warps work
-        return s->grp_rows <= 32 ? attn_windowed_d<D, 32>(s, Kc, Vc, n_rows) : attn_windowed_d<D, 64>(s, Kc, Vc, n_rows);
+        // groups of at most 32 rows: every warp takes half of a key tile, so all four warps work;
+        // up to 64 rows: four warps of 16 queries; up to 128 rows: eight
+        if (s->grp_rows <= 32) return attn_windowed_d<D, 32, 4>(s, Kc, Vc, n_rows);
+        if (s->grp_rows <= 64) return attn_windowed_d<D, 64, 4>(s, Kc, Vc, n_rows);
+        return attn_windowed_d<D, 64, 8>(s, Kc, Vc, n_rows);
     }
     static int attn_windowed(rd_session* s, const void* Kc, const void* Vc, int n_rows) {
         switch (s->m->cfg.head_dim) {
@@ -743,7 +788,11 @@ template <typename T> struct Eng {
         LAUNCH(s, delta_kernel, n, DELTA_THREADS, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
         SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
         LAUNCH(s, advance_kernel, (B + 63) / 64, 64, 0, st, s->delta, B, s->sc.max_window, window, inner, eps,
-               s->sc.max_iters_per_pos, s->sc.max_new_tokens);
+               s->sc.max_iters_per_pos, s->sc.max_new_tokens, c.n_prelude + c.n_coda + inner * c.n_core);
+        // every weight matrix is streamed once per pass: prelude, coda and head once, core and adapter `inner` times
+        const uint64_t per_layer = 4ull * h * h + 3ull * h * c.mlp_inner;
+        s->stats.weight_bytes += ((uint64_t)(c.n_prelude + c.n_coda) * per_layer + (uint64_t)c.vocab * h +
+                                  (uint64_t)inner * (c.n_core * per_layer + 2ull * h * h)) * s->m->esz;
         return RD_OK;
     }
 
@@ -777,37 +826,23 @@ template <typename T> struct Eng {
         return RD_OK;
     }
 
+    // Enqueues the whole prefill on the session's stream and returns: the prompt goes through a pinned
+    // copy of its own, e and the latents of the prompt rows live in the session's workspace, and the
+    // sequence's state is set by a kernel behind the passes.
     static int prefill(rd_session* s, int seq, const int32_t* prompt, int L, int r) {
-        const int h = s->m->cfg.hidden;
-        CU(cudaStreamSynchronize(s->stream));
-        CU(cudaMemcpy(s->tokens + (size_t)seq * s->tok_stride, prompt, (size_t)L * sizeof(int), cudaMemcpyHostToDevice));
+        const int buf = s->stage_next;
+        CU(cudaEventSynchronize(s->prompt_ev[buf]));      // the upload that last used this copy has finished
+        memcpy(s->prompt_stage[buf], prompt, (size_t)L * sizeof(int));
+        CU(cudaMemcpyAsync(s->tokens + (size_t)seq * s->tok_stride, s->prompt_stage[buf], (size_t)L * sizeof(int),
+                           cudaMemcpyHostToDevice, s->stream));
+        CU(cudaEventRecord(s->prompt_ev[buf], s->stream));
+        s->stage_next = (buf + 1) % rd_session::PROMPT_STAGES;
         const int n = L - 1;   // rows 0..L-2 are prefilled; L-1 is the first in-flight row
-        float *e_all = nullptr, *s_all = nullptr;
-        int rc = RD_OK;
-        if (n > 0) {
-            RD_TRY(s->mem.get(&e_all, (size_t)n * h * sizeof(float)));
-            rc = s->mem.get(&s_all, (size_t)n * h * sizeof(float));
-            if (!rc) rc = prefill_passes(s, seq, n, r, e_all, s_all);
-        }
-        if (!rc) {
-            cudaError_t e = cudaStreamSynchronize(s->stream);
-            if (e == cudaSuccess) e = cudaGetLastError();
-            if (e != cudaSuccess) rc = cuda_fail(e, "prefill", __LINE__);
-        } else {
-            cudaStreamSynchronize(s->stream);
-        }
-        if (e_all) s->mem.release(e_all);
-        if (s_all) s->mem.release(s_all);
-        if (rc) return rc;
+        if (n > 0) RD_TRY(prefill_passes(s, seq, n, r, s->pf_e, s->pf_s));
         // sequence state: |y_frozen| = L, one fresh in-flight row at position L-1
-        const int one = 1, zero = 0, isdone = s->sc.max_new_tokens <= 0 ? 1 : 0;
+        SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
         const int slot = seq * s->sc.max_window + (L - 1) % s->sc.max_window;
-        CU(cudaMemcpy(s->n_prompt + seq, &L, sizeof(int), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(s->n_committed + seq, &L, sizeof(int), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(s->win_len + seq, isdone ? &zero : &one, sizeof(int), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(s->done + seq, &isdone, sizeof(int), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(s->row_steps + slot, &zero, sizeof(int), cudaMemcpyHostToDevice));
-        CU(cudaMemcpy(s->row_iters + slot, &zero, sizeof(int), cudaMemcpyHostToDevice));
+        LAUNCH(s, seq_start_kernel, 1, 32, 0, st, seq, L, slot, s->sc.max_new_tokens <= 0 ? 1 : 0);
         return RD_OK;
     }
 };
@@ -943,7 +978,7 @@ extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int
                                 int32_t n, float* dst) {
     if (!s || !dst || block < 0 || block > 2 || (which != 0 && which != 1) || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
     const rd_config& c = s->m->cfg;
-    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 + n > s->sc.max_context) return RD_E_INVALID_ARG;
+    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 > s->sc.max_context || n > s->sc.max_context - pos0) return RD_E_INVALID_ARG;
     RD_TRY(rd_sync(s));
     if (n == 0) return RD_OK;
     const size_t off = ((size_t)layer * s->sc.batch + seq) * s->seq_stride;
@@ -974,7 +1009,6 @@ extern "C" int rd_debug_read_kv(rd_session* s, int32_t block, int32_t layer, int
 // ---------------------------------------------------------------------------------------------
 constexpr size_t RD_KV_STAGE_ELEMS = (size_t)1 << 20;
 static __device__ __align__(256) float g_kv_stage[RD_KV_STAGE_ELEMS];
-constexpr int RD_MAX_DEVICES = 64;
 static float* g_kv_stage_dev[RD_MAX_DEVICES];
 static std::mutex g_kv_stage_mutex;
 
@@ -996,7 +1030,7 @@ extern "C" int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t la
                                         int32_t pos0, int32_t n, float* dst) {
     if (!s || !dst || block < 0 || block > 2 || (which != 0 && which != 1) || seq < 0 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
     const rd_config& c = s->m->cfg;
-    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 + n > s->sc.max_context) return RD_E_INVALID_ARG;
+    if (layer < 0 || layer >= n_layers_of(c, block) || pos0 < 0 || n < 0 || pos0 > s->sc.max_context || n > s->sc.max_context - pos0) return RD_E_INVALID_ARG;
     const size_t cnt = (size_t)n * c.hidden;
     if (cnt > RD_KV_STAGE_ELEMS) {
         snprintf(g_cuda_err, sizeof g_cuda_err,
@@ -1027,13 +1061,27 @@ extern "C" int rd_debug_read_kv_noalloc(rd_session* s, int32_t block, int32_t la
 extern "C" int rd_stats(rd_session* s, rd_stats_t* out) {
     if (!s || !out) return RD_E_INVALID_ARG;
     RD_TRY(rd_sync(s));
-    unsigned long long cnt[8];
+    unsigned long long cnt[RD_COUNTERS];
     CU(cudaMemcpy(cnt, s->counters, sizeof cnt, cudaMemcpyDeviceToHost));
     *out = s->stats;
     out->rows_prelude = cnt[0];
     out->rows_core = cnt[1];
     out->rows_coda = cnt[2];
     out->tokens_committed = cnt[3];
+    const rd_config& c = s->m->cfg;
+    const uint64_t h = c.hidden, per_layer = 4 * h * h + 3 * h * (uint64_t)c.mlp_inner;
+    const uint64_t rows_written = cnt[0] * c.n_prelude + cnt[1] * c.n_core + cnt[2] * c.n_coda;
+    out->kv_bytes = (cnt[4] + rows_written) * 2 * h * s->m->esz;
+    out->flops = 2 * (cnt[0] * c.n_prelude * per_layer + cnt[1] * (c.n_core * per_layer + 2 * h * h) +
+                      cnt[2] * (c.n_coda * per_layer + (uint64_t)c.vocab * h)) + 4 * h * cnt[5];
+    for (int k = 0; k < RD_HIST_BINS; k++) out->commit_hist[k] = cnt[RD_HIST_AT + k];
+    return RD_OK;
+}
+
+extern "C" int rd_debug_expire_next_wait(rd_session* s) {
+    if (!s) return RD_E_INVALID_ARG;
+    if (!(s->gemm_path >= 1 && s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
+    s->expire_next_wait = true;
     return RD_OK;
 }
 

@@ -62,7 +62,7 @@ def from_bf16_bits(b: np.ndarray) -> np.ndarray:
 
 
 def make_weights(hidden, mlp_inner, n_prelude, n_core, n_coda, vocab, tie_embeddings=True,
-                 seed=0, std=0.02, gain_jitter=0.0, bf16=False, adapter_s_scale=1.0):
+                 seed=0, std=0.02, gain_jitter=0.0, bf16=False, adapter_s_scale=1.0, layer_scale=1.0):
     """Random-init weights: matrices N(0, std), gains 1 + gain_jitter * N(0,1).
 
     Returns a dict name -> float32 array in `tensor_specs` order.  With
@@ -70,7 +70,10 @@ def make_weights(hidden, mlp_inner, n_prelude, n_core, n_coda, vocab, tie_embedd
     stay float32), so both consumers see exactly the values the bf16
     configuration stores.  `adapter_s_scale` scales the half of the adapter
     that multiplies the latent state (columns h..2h-1); tests use it to make
-    the recurrence more or less contractive.
+    the recurrence more or less contractive.  `layer_scale` scales every
+    matrix inside the layers (wq .. wd; not the embedding, adapter or head):
+    below 1 a layer adds less to its residual stream, so it amplifies
+    perturbations of its input less.
     """
     rng = np.random.default_rng(seed)
     out = {}
@@ -86,6 +89,8 @@ def make_weights(hidden, mlp_inner, n_prelude, n_core, n_coda, vocab, tie_embedd
         w *= np.float32(std)
         if name == "adapter" and adapter_s_scale != 1.0:
             w[:, hidden:] *= np.float32(adapter_s_scale)
+        if layer_scale != 1.0 and "." in name:
+            w *= np.float32(layer_scale)
         if bf16:
             w = from_bf16_bits(to_bf16_bits(w))
         out[name] = w

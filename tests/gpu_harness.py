@@ -39,7 +39,7 @@ class LockStep:
     token w with u(w) < top_p - nucleus_band beats g's score by more than tie_gap."""
 
     def __init__(self, sampler: orc.Sampler, session: rd.Session, seqs, tol: Tolerance, tie_gap=0.0,
-                 check_logits=True, logit_noise=None, nucleus_band=0.0):
+                 check_logits=True, logit_noise=None, nucleus_band=0.0, delta_tol=None):
         """logit_noise = (rms, fraction, max_abs): instead of bounding every logit by `tol`, bound the
         rms error, the fraction of logits outside `tol` and the largest error (used at the full
         3.5B widths, where bf16 rounding noise amplified by the random-init layers puts a few
@@ -48,10 +48,20 @@ class LockStep:
         self.check_logits = check_logits
         self.logit_noise = logit_noise
         self.nucleus_band = nucleus_band
+        # Eq. 3: |delta_gpu - delta_oracle| <= abs + rel * max(delta_oracle, 1e-6).  Latents that agree
+        # within t per element give deltas that agree within 2 t (1 + delta) at worst (the norms of z
+        # and of z - z_prev each move by at most t sqrt(h), and ||z|| ~ sqrt(h) after the closing
+        # RMSNorm).  float32 configuration (t = 1e-4 stated, a few 1e-6 in practice): 2e-5 + 1e-3 delta,
+        # ten times inside that worst case; bf16: the stated 5e-2 + 2e-2 |want| applied to delta itself.
+        # Independently of the latents' error, the kernel's own arithmetic is checked to 2e-5 relative
+        # against Eq. 3 evaluated on the GPU's own latents (below).
+        self.delta_tol = delta_tol if delta_tol is not None else ((2e-5, 1e-3) if tol.abs_tol <= 1e-3 else (tol.abs_tol, tol.rel_tol))
+        self.gpu_z_prev = {}            # (sequence, position) -> the GPU's latent after the previous step
+        self._seq_seen = {}             # sequence slot -> the oracle's Sequence object those latents belong to
         self.near_ties = 0
         self.boundary_cases = 0
         self.n_drafts = 0
-        self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0}
+        self.max_err = {"z": 0.0, "logits": 0.0, "delta": 0.0, "delta_rel": 0.0, "delta_kernel_rel": 0.0}
         self.steps = 0
 
     def _scores(self, logits, sq, token_pos):
@@ -75,6 +85,10 @@ class LockStep:
         self.steps += 1
         for sq, info in zip(self.seqs, infos):
             b = sq.seq_id
+            if self._seq_seen.get(b) is not sq:          # a new request in this slot: forget the old latents
+                self._seq_seen[b] = sq
+                for key in [k for k in self.gpu_z_prev if k[0] == b]:
+                    del self.gpu_z_prev[key]
             if info is None:
                 continue
             f, n = self.sess.last_step_rows(b)
@@ -98,9 +112,34 @@ class LockStep:
                         f"step {self.steps} seq {b}: logits rms err {rms:.3e}, outside tolerance {frac:.3%}, max {err.max():.3e}"
             if delta_checked and "delta" in info:
                 dl = self.sess.debug_read(rd.RD_DBG_DELTA, b)
-                fin = np.isfinite(info["delta"])
+                want = info["delta"]
+                fin = np.isfinite(want)
+                assert np.array_equal(np.isfinite(dl), fin), f"step {self.steps} seq {b}: delta finiteness differs"
                 if fin.any():
-                    self.max_err["delta"] = max(self.max_err["delta"], float(np.abs(dl - info["delta"])[fin].max()))
+                    err = np.abs(dl - want)[fin]
+                    ref = np.maximum(want[fin], 1e-6)
+                    self.max_err["delta"] = max(self.max_err["delta"], float(err.max()))
+                    self.max_err["delta_rel"] = max(self.max_err["delta_rel"], float((err / ref).max()))
+                    bound = self.delta_tol[0] + self.delta_tol[1] * ref
+                    assert (err <= bound).all(), \
+                        f"step {self.steps} seq {b}: delta (Eq. 3) off by {err.max():.3e} (relative {(err / ref).max():.3e}), GPU {dl} vs oracle {want}"
+                # the kernel alone: Eq. 3 evaluated here (float64) on the GPU's own latents of this
+                # step and of the step before (a fresh row starts from its initial state)
+                for i in range(n):
+                    key = (b, int(info["pos"][i]))
+                    zp = self.gpu_z_prev.get(key)
+                    if zp is None:
+                        c = self.sm.m.cfg
+                        zp = orc.init_state(self.sm.seed, b, key[1], c.hidden, c.init_sigma, np.float64).astype(np.float32)
+                    zi = z[i].astype(np.float64)
+                    den = np.sqrt(np.sum(zi * zi))
+                    if den > 0 and np.isfinite(dl[i]):
+                        want_k = np.sqrt(np.sum((zi - zp.astype(np.float64)) ** 2)) / den
+                        rel = abs(float(dl[i]) - want_k) / max(want_k, 1e-6)
+                        self.max_err["delta_kernel_rel"] = max(self.max_err["delta_kernel_rel"], rel)
+                        assert rel <= 2e-5, f"step {self.steps} seq {b} row {i}: delta kernel {dl[i]:.8e} vs {want_k:.8e} from the GPU's own latents"
+            for i in range(n):
+                self.gpu_z_prev[(b, int(info["pos"][i]))] = z[i].copy()
             drafts = self.sess.debug_read(rd.RD_DBG_DRAFTS, b)
             self.n_drafts += n
             for i in range(n):

@@ -172,3 +172,54 @@ def test_twin_batch_16_window_16_is_256_rows(path):
         ls.df(16, 1, 1e-3)
     assert _ties_ok(ls)
     assert sess.stats()["tc_gemm_launches"] > 0      # no silent fall-back to the plain kernels
+
+
+def test_twin_window_64_rows_plain_init_first_steps():
+    """The 64-row window with the plain random init (no scaling of the adapter): the first 16 steps,
+    before rounding differences have had many recurrences to grow."""
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 64, 70, max_ctx=256)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [50], 2, 70)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    for _ in range(16):
+        ls.df(64, 1, 0.0)
+    assert len(seqs[0].window) == 17 and _ties_ok(ls)
+
+
+@pytest.mark.parametrize("scale,steps", [(0.25, 140), (1.0, 16)])
+def test_twin_window_128_rows(scale, steps):
+    """The paper's default maximum wavefront, 128 rows of one sequence: the eight-warp attention
+    groups and the 128-row GEMM tile.  The full ramp runs with the contractive adapter (a row stays in
+    flight for 128 recurrences), the plain init for the first 16 steps."""
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 128, 140, max_ctx=256, adapter_s_scale=scale)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, [40], 2, 140)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    widest = 0
+    for _ in range(steps):
+        if ls.all_done():
+            break
+        ls.df(128, 1, 0.0)
+        widest = max(widest, len(seqs[0].window))
+    assert widest == min(128, steps + 1)
+    assert _ties_ok(ls)
+    assert sess.stats()["tc_gemm_launches"] > 0
+
+
+def test_twin_long_context_batch_4_window_32():
+    """The long-context regime: four sequences with prompts of about 4,100 tokens (ragged), a 32-row
+    wavefront each (128 rows per step), greedy.  Every head's keys span 65 tiles, cut into 8 splits
+    per (sequence, head), and the prefill runs in nine 512-row chunks per sequence."""
+    lens = [4096, 4033, 4127, 3970]
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, 32, 36, batch=4, max_ctx=4200)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 1, 36)
+    # cache rows of the prefill, deep inside the prefix and at its end
+    for b, L in ((0, 4096), (3, 3970)):
+        for blk, name in enumerate(("prelude", "core", "coda")):
+            got = sess.read_kv(blk, 1, 0, b, L - 70, 69)
+            want = seqs[b].caches[name].K[1, L - 70:L - 1].reshape(69, -1)
+            assert TOL.excess(got, want) <= 0, f"sequence {b} {name} keys off by {np.abs(got - want).max():.3e}"
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    for _ in range(34):
+        ls.df(32, 1, 0.0)
+    assert all(len(sq.window) == 32 for sq in seqs)
+    print(f"near-ties {ls.near_ties} of {ls.n_drafts}, max err {ls.max_err}")
+    assert _ties_ok(ls)

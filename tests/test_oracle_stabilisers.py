@@ -53,9 +53,61 @@ def test_momentum_is_the_stated_recursion_per_position():
                 assert np.allclose(got[p], e_hist[p], rtol=0, atol=1e-12)
 
 
-def test_noise_schedule_is_linear_and_ends_at_zero():
-    """With beta = 1 a position's first step starts from pure noise (its initial state is wiped out),
-    and at step t the mix is beta (1 - t / T)."""
+def _check_noise_mix_against_hand_schedule(W, inner, eps, cap, schedule, n_steps):
+    """Every step: recompute z = R^inner(e, (1 - b) z + b z_noise) from each row's stored z and the
+    number of steps it has taken, with b read from `schedule` (numbers, not the formula), on a copy
+    of the caches, and compare with what the sampler produced."""
+    import copy
+    beta = 0.8
+    model, _ = make_oracle(SMALL, seed=1)
+    sm = orc.Sampler(model, seed=3, beta=beta, max_iters_per_pos=cap)
+    sq = sm.prefill(0, rd_inputs.make_prompt(9, SMALL["vocab"], seed=2), 2, 12)
+    seen = set()
+    for _ in range(n_steps):
+        rows = sq.window
+        pos = np.array([r.pos for r in rows])
+        caches = copy.deepcopy(sq.caches)
+        e = model.prelude(sq.tokens[pos], pos, caches)
+        z = np.stack([r.z for r in rows]).copy()
+        for i, r in enumerate(rows):
+            b = schedule[r.steps]
+            seen.add(r.steps)
+            noise = orc.latent_noise(3, 0, r.pos, r.steps, SMALL["hidden"], 1.0, model.dtype)
+            z[i] = (1.0 - b) * z[i] + b * noise
+        for _ in range(inner):
+            z = model.core(e, z, pos, caches)
+        info = sm.df_step(sq, W, inner, eps)
+        assert np.allclose(info["z"], z, rtol=0, atol=1e-6), f"rows at steps {[r.steps - 1 for r in rows]}"
+    return seen
+
+
+def test_noise_schedule_fixed_exit_is_the_hand_written_one():
+    """Fixed exit, window 4, beta 0.8: a position's steps 0, 1, 2, 3 mix in 0.8, 0.6, 0.4, 0.2 of noise
+    (linear in the steps taken, the later steps less noisy; zero would come at step 4, which no
+    position takes)."""
+    seen = _check_noise_mix_against_hand_schedule(4, 1, 0.0, 64, {0: 0.8, 1: 0.6, 2: 0.4, 3: 0.2}, 8)
+    assert seen == {0, 1, 2, 3}
+
+
+def test_noise_schedule_adaptive_exit_runs_over_cap_by_inner_steps():
+    """Adaptive exit, cap 12 core iterations, 2 per step: a position gets 6 steps and its mix falls
+    from 0.8 by 0.8 / 6 per step."""
+    sched = {0: 0.8, 1: 0.6666666666666667, 2: 0.5333333333333333, 3: 0.4, 4: 0.26666666666666666, 5: 0.13333333333333333}
+    seen = _check_noise_mix_against_hand_schedule(8, 2, 1e-12, 12, sched, 9)
+    assert seen == {0, 1, 2, 3, 4, 5}
+
+
+def test_a_shifted_or_shortened_schedule_is_told_apart():
+    """The check above has teeth: schedules off by one step, or stretched over one step fewer, miss
+    by far more than its tolerance."""
+    import pytest
+    for wrong in ({0: 0.6, 1: 0.4, 2: 0.2, 3: 0.0}, {0: 0.8, 1: 0.8 * 2 / 3, 2: 0.8 / 3, 3: 0.0}):
+        with pytest.raises(AssertionError):
+            _check_noise_mix_against_hand_schedule(4, 1, 0.0, 64, wrong, 8)
+
+
+def test_full_strength_noise_wipes_out_the_initial_state():
+    """With beta = 1 a position's first step starts from pure noise."""
     model, _ = make_oracle(SMALL, seed=1)
     W = 4
     sm = orc.Sampler(model, seed=3, beta=1.0)
@@ -69,9 +121,6 @@ def test_noise_schedule_is_linear_and_ends_at_zero():
     info = sm.df_step(sq, W, 1, 0.0)
     assert np.allclose(info["z"][0], want[0], atol=1e-12)
     assert not np.allclose(noise0, z0)
-    # schedule values through the public behaviour: beta_t for t = 0..T
-    betas = [0.8 * max(0.0, 1.0 - t / W) for t in range(W + 1)]
-    assert betas[0] == 0.8 and betas[-1] == 0.0 and np.allclose(np.diff(betas), -0.2)
 
 
 def test_noise_draws_are_fresh_per_step_and_standard_normal():
