@@ -13,9 +13,10 @@ def oracle_config(shape, **kw):
 
 
 def make_oracle(shape, seed=0, std=0.02, gain_jitter=0.1, dtype=np.float64, contract=False,
-                bf16=False, max_ctx=256, adapter_s_scale=1.0, **cfg_kw):
+                bf16=False, max_ctx=256, adapter_s_scale=1.0, layer_scale=1.0, **cfg_kw):
     w = rd_inputs.make_weights(**rd_inputs.shape_args(shape), seed=seed, std=std,
-                               gain_jitter=gain_jitter, bf16=bf16, adapter_s_scale=adapter_s_scale)
+                               gain_jitter=gain_jitter, bf16=bf16, adapter_s_scale=adapter_s_scale,
+                               layer_scale=layer_scale)
     model = orc.RDModel(oracle_config(shape, **cfg_kw), w, dtype=dtype, contract=contract,
                         max_ctx=max_ctx)
     return model, w
