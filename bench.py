@@ -289,9 +289,14 @@ def run_ours(args):
     pinned = [torch.from_numpy(p).pin_memory() for p in prompts]
 
     def new_session(window, temperature=0.0):
-        return rd.Session(model, batch=B, max_context=max_ctx, max_window=window, max_iters_per_pos=64,
-                          max_new_tokens=N, temperature=temperature, seed=1234, stream=stream.cuda_stream,
-                          top_p=wl.get("top_p", 0.0))
+        ses = rd.Session(model, batch=B, max_context=max_ctx, max_window=window, max_iters_per_pos=64,
+                         max_new_tokens=N, temperature=temperature, seed=1234, stream=stream.cuda_stream,
+                         top_p=wl.get("top_p", 0.0))
+        if args.unfused_swiglu:
+            ses.set_fused_swiglu(False)     # A/B: gate/up leaves partial sums, SwiGLU in a kernel of its own
+        if args.unchained:
+            ses.set_launch_chaining(False)  # A/B: ordinary stream-ordered launches
+        return ses
 
     def prefill(sess):
         for b in range(B):
@@ -489,7 +494,8 @@ def run_ours(args):
                    "inner_iters": wl["inner"], "exit_threshold": wl["eps"], "ar_r": wl["ar_r"],
                    "temperature": wl["temperature"], "top_p": wl.get("top_p", 0.0),
                    "l2": "inputs larger than L2 (weights streamed per step: %.2f GB)" % (step_b / 1e9),
-                   "multi_gpu": "replicas only (no data-path collective)"},
+                   "multi_gpu": "replicas only (no data-path collective)",
+                   "variant": {"fused_swiglu": not args.unfused_swiglu, "chained_launches": not args.unchained}},
         "df_tok_s": df_tok_s, "ar_tok_s": ar_tok_s, "df_over_ar": df_tok_s / ar_tok_s if ar_tok_s else None,
         "ar_tokens_timed": n_ar, "ar_ms_per_token": ar_ms / n_ar,
         "prefill": {"seconds": prefill_s, "flops": pf_flops, "tflops": pf_flops / prefill_s / 1e12,
@@ -637,6 +643,8 @@ def main():
     ap.add_argument("--temperature", type=float, default=-1.0, help="override the workload's sampling temperature (sweeps)")
     ap.add_argument("--top-p", type=float, default=0.0, help="top-p of Sample (sweeps; needs a temperature > 0)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused-swiglu", action="store_true", help="A/B: SwiGLU as a separate kernel")
+    ap.add_argument("--unchained", action="store_true", help="A/B: no programmatic dependent launch")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
     if args.impl == "reference":

@@ -257,6 +257,12 @@ int rd_set_gemm_path(rd_session* s, int32_t path);
  * 0: ordinary stream-ordered launches.  Results are identical; for measurement and tests. */
 int rd_set_launch_chaining(rd_session* s, int32_t on);
 
+/* rd_set_fused_swiglu -- 1 (default): on the tensor-core path the gate/up projection runs on whole
+ * tiles and its epilogue writes silu(gate) * up directly (no partial sums, no separate kernel);
+ * 0: the projection leaves partial sums and a separate kernel applies the SwiGLU.  Same arithmetic up
+ * to the order of the float32 sums; for measurement (A/B) and tests. */
+int rd_set_fused_swiglu(rd_session* s, int32_t on);
+
 const char* rd_strerror(int code);
 /* Text of the last CUDA error this library saw on the calling thread's most recent failing call
  * (static storage, never NULL). */

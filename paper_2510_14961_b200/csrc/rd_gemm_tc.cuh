@@ -55,6 +55,11 @@ constexpr int TC_BK = 64;        // k per stage: 64 bf16 = one 128-byte swizzle 
 constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
 
+struct TcParamsFuse {
+    __nv_bfloat16* act_out;
+    int act_ld, n_rows, inner;
+};
+
 struct TcWeight {
     CUtensorMap map;             // box of 128 output features
     CUtensorMap map2;            // box of 256 output features (two tiles per unit, see TC_MT)
@@ -256,6 +261,24 @@ __host__ __device__ constexpr uint32_t umma_idesc(int bn, int m = TC_BM) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// SwiGLU on 32 accumulator columns (= rows) of this lane's feature.  Lanes 2i and 2i+1 hold gate i and
+// up i of the same inner feature; the pair splits the columns between them (even lane: even columns,
+// odd lane: odd columns), so every lane computes and stores 16 values.
+//   raw: 32 columns of this lane; row0: row of column 0; feat: inner feature of the lane pair.
+__device__ __forceinline__ void swiglu_store32(const uint32_t* raw, int lane, int row0, int feat, const TcParamsFuse& f) {
+    const bool odd = lane & 1;
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) {
+        const float a = __uint_as_float(raw[j]), b = __uint_as_float(raw[j + 1]);
+        const float got = __shfl_xor_sync(0xffffffffu, odd ? a : b, 1);
+        const float g = odd ? got : a;            // even lane: its own gate of column j; odd lane: the partner's gate of column j+1
+        const float u = odd ? b : got;
+        const int row = row0 + j + (odd ? 1 : 0);
+        if (row < f.n_rows && feat < f.inner)
+            f.act_out[(size_t)row * f.act_ld + feat] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
+    }
+}
+
 #ifndef RD_TC_RING_KB
 #define RD_TC_RING_KB 100
 #endif
@@ -294,6 +317,10 @@ struct TcParams {
     int max_seg;               // scratch slots per CTA
     float* scratch;            // [gridDim.x * max_seg][MT][BN][128] partial sums
     int* status;
+    // Fused SwiGLU epilogue (gate/up projection with rows interleaved: feature 2j = gate j, 2j+1 = up j).
+    // Non-null act_out: every CTA's share is whole tiles (per is a multiple of kb), nothing goes to the
+    // scratch buffer, and the epilogue writes silu(gate) * up as bf16 to act_out[row * act_ld + j].
+    TcParamsFuse fuse;         // fuse.act_out; rows >= fuse.n_rows and inner features >= fuse.inner are not written
     uint32_t spin_limit;       // polls a wait on a pipeline barrier may take (TC_SPIN_LIMIT)
     int skip_unit;             // -1.  Test aid (rd_debug_expire_next_wait): CTA 0's producer leaves this unit of
                                // its share out, so that the barrier the unit would complete is never completed
@@ -425,7 +452,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const uint32_t t = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * C::MT * C::ACC_COLS);
                 // the share's seg-th segment (= seg-th tile it touches) -> slot blockIdx.x * max_seg + seg
                 float* slot = p.scratch + ((size_t)blockIdx.x * p.max_seg + seg) * (size_t)(C::MT * BN * TC_BM) + quad * 32 + lane;
-                if constexpr (BN >= 32) {
+                if (p.fuse.act_out) {
+                    // whole tile (ka == 0, len == kb): SwiGLU straight from the accumulator
+                    const int tile = (int)(u / p.kb);
+                    const int ftu = tile / p.n_tiles_n, rt = tile % p.n_tiles_n;
+                    if constexpr (BN >= 32) {
+#pragma unroll 1
+                        for (int c = 0; c < C::MT * BN; c += 32) {
+                            uint32_t raw[32];
+                            tmem_ld32(t + (uint32_t)((c / BN) * C::ACC_COLS + c % BN), raw);
+                            const int feat = ((ftu * C::MT + c / BN) * TC_BM + quad * 32 + lane) >> 1;
+                            swiglu_store32(raw, lane, rt * BN + c % BN, feat, p.fuse);
+                        }
+                    } else {
+                        uint32_t raw[32];
+                        tmem_ld16(t, raw);
+#pragma unroll
+                        for (int j = 16; j < 32; j++) raw[j] = 0;
+                        TcParamsFuse f16 = p.fuse;
+                        f16.n_rows = min(f16.n_rows, rt * BN + 16);          // columns 16.. do not exist
+                        swiglu_store32(raw, lane, rt * BN, ((ftu * TC_BM) + quad * 32 + lane) >> 1, f16);
+                    }
+                } else if constexpr (BN >= 32) {
 #pragma unroll 1
                     for (int c = 0; c < C::MT * BN; c += 32) {  // column c = (feature tile in the unit) * BN + row
                         uint32_t raw[32];
@@ -630,12 +678,25 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 // slot of the pair's seg-th segment; this CTA's feature tile is the rank-th of the unit's two
                 float* slot = p.scratch + ((size_t)pair * p.max_seg + seg) * (size_t)(2 * C::BN * TC_BM) +
                               (size_t)rank * (C::BN * TC_BM) + quad * 32 + lane;
+                if (p.fuse.act_out) {
+                    // whole tile: SwiGLU straight from this CTA's 128 features of the accumulator
+                    const int tile = (int)(u / p.kb);
+                    const int ft = (tile / p.n_tiles_n) * 2 + (int)rank, rt = tile % p.n_tiles_n;
+                    const int feat = (ft * TC_BM + quad * 32 + lane) >> 1;
 #pragma unroll 1
-                for (int c = 0; c < C::BN; c += 32) {
-                    uint32_t raw[32];
-                    tmem_ld32(t + (uint32_t)c, raw);
+                    for (int c = 0; c < C::BN; c += 32) {
+                        uint32_t raw[32];
+                        tmem_ld32(t + (uint32_t)c, raw);
+                        swiglu_store32(raw, lane, rt * C::BN + c, feat, p.fuse);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int c = 0; c < C::BN; c += 32) {
+                        uint32_t raw[32];
+                        tmem_ld32(t + (uint32_t)c, raw);
 #pragma unroll
-                    for (int j = 0; j < 32; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
+                        for (int j = 0; j < 32; j++) slot[(size_t)(c + j) * TC_BM] = __uint_as_float(raw[j]);
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -673,7 +734,8 @@ struct TcPlan {
 // Every CTA gets `per` consecutive units (the last ones possibly fewer).
 // `pair`: tiles of 128 and 256 rows go to CTA pairs (gemm_tc_pair_kernel) instead of single CTAs.
 constexpr int TC_PAIR_MIN_BN = 128;
-static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair = true) {
+// `whole_tiles`: a share is a whole number of tiles (for the fused SwiGLU epilogue, which needs finished sums).
+static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair = true, bool whole_tiles = false) {
     TcPlan pl;
     pl.bn_idx = tc_pick_bn(n_rows);
     pl.bn = 16 << pl.bn_idx;
@@ -687,6 +749,11 @@ static inline TcPlan tc_plan(int K, int n_out, int n_rows, int n_sms, bool pair 
     pl.units = (long long)pl.n_tiles_m * pl.n_tiles_n * pl.kb;
     const long long g = std::min<long long>(n_sms, pl.units);
     pl.per = (int)((pl.units + g - 1) / g);
+    if (whole_tiles) {
+        const long long tiles = (long long)pl.n_tiles_m * pl.n_tiles_n;
+        const long long gt = std::min<long long>(n_sms, tiles);
+        pl.per = (int)((tiles + gt - 1) / gt) * pl.kb;
+    }
     pl.grid = (int)((pl.units + pl.per - 1) / pl.per);
     pl.max_seg = (pl.per + pl.kb - 1) / pl.kb + 1;      // tiles a run of `per` units can touch
     pl.scratch_elems = (size_t)pl.grid * pl.max_seg * pl.mt * pl.bn * TC_BM;
@@ -726,13 +793,14 @@ static inline int tc_configure_device() {
 // the shape is not taken (caller falls back to the SIMT kernels).
 static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, int K, int n_out, int n_rows,
                           float* scratch, size_t scratch_elems, int n_sms, int* status, bool chained, PartialSums* out,
-                          bool pair = true, bool* expire_wait = nullptr) {
+                          bool pair = true, bool* expire_wait = nullptr, const TcParamsFuse* fuse = nullptr) {
     if (ta.K != K || tw.K != K || tw.n_out != n_out || n_rows < 1 || n_rows > ta.rows) return RD_E_INVALID_ARG;
-    const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms, pair);
-    if (pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
+    const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms, pair, fuse != nullptr);
+    if (!fuse && pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
     p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
     p.scratch = scratch; p.status = status;
+    p.fuse = fuse ? *fuse : TcParamsFuse{nullptr, 0, 0, 0};
     p.spin_limit = TC_SPIN_LIMIT; p.skip_unit = -1;
     if (expire_wait && *expire_wait && !pl.pair) {
         // test aid, one launch: CTA 0 never loads the first unit of its share and every wait of the

@@ -494,27 +494,50 @@ attn_row_kernel(const T* __restrict__ q_t, const int* __restrict__ row_pos, cons
     }
 }
 
-// act[r, j..j+3] = silu(gate) * up with gate = acc[r, j], up = acc[r, I + j] of the gate/up GEMM.
+// act[r, j..j+3] = silu(gate) * up of the gate/up GEMM's result.  Stacked layout: gate j = acc[r, j],
+// up j = acc[r, I + j].  Interleaved layout (models whose gate/up matrix was interleaved at load for
+// the fused tensor-core epilogue): gate j = acc[r, 2j], up j = acc[r, 2j + 1].
 template <typename T>
 __global__ void swiglu_kernel(const RowSource src, int inner, T* __restrict__ act, size_t lda, int n_rows,
-                              const int* __restrict__ row_pos) {
+                              const int* __restrict__ row_pos, int interleaved) {
     pdl_trigger();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t quads = (size_t)inner / 4;
     const bool mine = i < (size_t)n_rows * quads;
     const int r = mine ? (int)(i / quads) : 0, j = mine ? (int)(i % quads) * 4 : 0;
-    // where the gate and up sums sit: arithmetic only, done before the wait for the GEMM
+    // where the sums sit: arithmetic only, done before the wait for the GEMM
     constexpr int NQ = 2;      // a gate/up tile is cut into at most 2 segments at the model shapes here
-    const RowSlots<NQ> sg = row_source_locate<NQ>(src, r, j), su = row_source_locate<NQ>(src, r, inner + j);
+    const int ma = interleaved ? 2 * j : j, mb = interleaved ? 2 * j + 4 : inner + j;
+    const RowSlots<NQ> sa = row_source_locate<NQ>(src, r, ma), sb = row_source_locate<NQ>(src, r, mb);
     pdl_wait();
     if (!mine) return;
-    const bool located = sg.n <= NQ && su.n <= NQ;
-    const float4 g = located ? row_source_fetch<NQ>(sg) : row_source_load4(src, r, j),
-                 u = located ? row_source_fetch<NQ>(su) : row_source_load4(src, r, inner + j);
+    const bool located = sa.n <= NQ && sb.n <= NQ;
+    const float4 a = located ? row_source_fetch<NQ>(sa) : row_source_load4(src, r, ma),
+                 b = located ? row_source_fetch<NQ>(sb) : row_source_load4(src, r, mb);
     if (row_pos[r] < 0) return;
-    const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+    float gv[4], uv[4];
+    if (interleaved) {
+        gv[0] = a.x; uv[0] = a.y; gv[1] = a.z; uv[1] = a.w;
+        gv[2] = b.x; uv[2] = b.y; gv[3] = b.z; uv[3] = b.w;
+    } else {
+        gv[0] = a.x; gv[1] = a.y; gv[2] = a.z; gv[3] = a.w;
+        uv[0] = b.x; uv[1] = b.y; uv[2] = b.z; uv[3] = b.w;
+    }
 #pragma unroll
     for (int k = 0; k < 4; k++) act[(size_t)r * lda + j + k] = from_f<T>((gv[k] / (1.0f + expf(-gv[k]))) * uv[k]);
+}
+
+// dst row 2j = gate row j, dst row 2j + 1 = up row j (rows of `cols` elements, 16-byte chunks).
+template <typename T>
+__global__ void interleave_rows_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ dst,
+                                       size_t inner, size_t cols) {
+    constexpr int VEC = 16 / sizeof(T);
+    const size_t chunks = cols / VEC, total = 2 * inner * chunks;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t row = i / chunks, c = i % chunks;
+        const T* src = (row & 1 ? up : gate) + (row >> 1) * cols + c * VEC;
+        *reinterpret_cast<uint4*>(dst + row * cols + c * VEC) = *reinterpret_cast<const uint4*>(src);
+    }
 }
 
 // Sample(p) of Algorithms 1-2 in two kernels.  Greedy: arg max, lowest index on ties.  Otherwise

@@ -94,6 +94,7 @@ struct rd_model {
     std::vector<LayerW> layers[3];
     TcWeight t_adapter, t_head;
     bool tc_ok = false;
+    bool gu_interleaved = false;   // gate/up matrices stored with rows interleaved (2j: gate j, 2j+1: up j)
     int n_sms = 148;
 };
 
@@ -126,6 +127,9 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
     size_t stage_n = 0;
     int rc = RD_OK;
     int idx = 0;
+    void* gu_tmp = nullptr;
+    // bf16 models that can take the tensor-core path store gate/up interleaved (hidden % 8 == 0 holds)
+    m->gu_interleaved = c.dtype == RD_BF16 && tc_init_driver() == RD_OK;
 
     auto mat = [&](void* dst, size_t n) -> int { return put_tensor(m, dst, t[idx++], n, elem_bytes, &stage, &stage_n); };
     auto gain = [&](float** dst) -> int {
@@ -147,8 +151,23 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
                 if ((rc = mat(L.wo, h * h))) break;
                 if ((rc = gain(&L.g2))) break;
                 if ((rc = m->mem.get(&L.wgu, 2 * I * h * es))) break;
-                if ((rc = mat(L.wgu, I * h))) break;
-                if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
+                if (m->gu_interleaved) {
+                    // gate and up land in a temporary and are woven row by row into the matrix the
+                    // fused tensor-core epilogue wants (one tile then holds both halves of a feature)
+                    if (!gu_tmp) {
+                        cudaError_t et = cudaMalloc(&gu_tmp, 2 * I * h * es);
+                        if (et != cudaSuccess) { rc = cuda_fail(et, "cudaMalloc", __LINE__); break; }
+                    }
+                    if ((rc = mat(gu_tmp, I * h))) break;
+                    if ((rc = mat((char*)gu_tmp + I * h * es, I * h))) break;
+                    interleave_rows_kernel<bf16><<<2048, 256>>>((const bf16*)gu_tmp, (const bf16*)gu_tmp + I * h, (bf16*)L.wgu, I, h);
+                    cudaError_t ek = cudaGetLastError();
+                    if (ek == cudaSuccess) ek = cudaDeviceSynchronize();
+                    if (ek != cudaSuccess) { rc = cuda_fail(ek, "interleave_rows_kernel", __LINE__); break; }
+                } else {
+                    if ((rc = mat(L.wgu, I * h))) break;
+                    if ((rc = mat((char*)L.wgu + I * h * es, I * h))) break;
+                }
                 if ((rc = m->mem.get(&L.wd, h * I * es))) break;
                 if ((rc = mat(L.wd, h * I))) break;
             }
@@ -166,6 +185,7 @@ static int load_impl(rd_model* m, const void* const* t, int elem_bytes) {
         }
     } while (0);
     if (stage) cudaFree(stage);
+    if (gu_tmp) cudaFree(gu_tmp);
     if (rc) return rc;
     // Tensor-core path: TMA descriptors over every weight matrix (bf16 only).
     m->tc_ok = false;
@@ -250,6 +270,7 @@ struct rd_session {
     bool expire_next_wait = false;            // test aid: see rd_debug_expire_next_wait
     float* acc = nullptr;          // output of the plain GEMM kernel, [rows, n_out]
     size_t acc_elems = 0;
+    bool fuse_swiglu = true;       // gate/up GEMM on whole tiles with the SwiGLU in its epilogue (tensor-core path)
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
@@ -507,6 +528,12 @@ extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
     return RD_OK;
 }
 
+extern "C" int rd_set_fused_swiglu(rd_session* s, int32_t on) {
+    if (!s || (on != 0 && on != 1)) return RD_E_INVALID_ARG;
+    s->fuse_swiglu = on != 0;
+    return RD_OK;
+}
+
 extern "C" int rd_set_launch_chaining(rd_session* s, int32_t on) {
     if (!s || (on != 0 && on != 1)) return RD_E_INVALID_ARG;
     s->chained = on != 0;
@@ -556,14 +583,20 @@ template <typename T> struct Eng {
 
     // acc[r, o] = sum_k A[r, k] W[o, k]; *out tells the consumer where the sums are: partial sums of
     // the tensor-core kernel, or the finished array s->acc of the plain kernel.
+    // With swiglu_out (gate/up projection of a model with interleaved gate/up rows) the tensor-core
+    // kernel finishes whole tiles and writes silu(gate) * up itself: *fused tells the caller so.
     static int gemm(rd_session* s, const T* A, size_t lda, const TcAct* ta, const T* W, const TcWeight* tw, int K,
-                    int n_out, int n_rows, RowSource* out) {
+                    int n_out, int n_rows, RowSource* out, T* swiglu_out = nullptr, bool* fused = nullptr) {
         const int br = bracket_open(s, 0, (uint64_t)n_out * K * sizeof(T));
         *out = RowSource{};
+        if (fused) *fused = false;
         if (tc_usable(s, ta, tw)) {
+            TcParamsFuse fz{(bf16*)swiglu_out, n_out / 2, n_rows, n_out / 2};
+            const bool fuse = swiglu_out != nullptr && fused != nullptr && s->m->gu_interleaved && s->fuse_swiglu;
             const int rc = tc_gemm(s->stream, *ta, *tw, K, n_out, n_rows, s->tc_scratch, s->tc_scratch_elems, s->m->n_sms,
-                                   s->status, s->chained, &out->part, s->gemm_path == 1, &s->expire_next_wait);
+                                   s->status, s->chained, &out->part, s->gemm_path == 1, &s->expire_next_wait, fuse ? &fz : nullptr);
             if (rc == RD_OK) {
+                if (fuse) *fused = true;
                 s->stats.tc_gemm_launches++; s->stats.kernel_launches++;
                 bracket_close(s, br);
                 return RD_OK;
@@ -675,9 +708,13 @@ template <typename T> struct Eng {
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, n_rows, &acc));
         Pending mid = {acc, x_in};                      // x_mid = x_in + out-projection, stored in s->x
         RD_TRY(norm<T>(s, mid, s->x, L.g2, (T*)s->act_h, n_rows));
-        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, n_rows, &acc));
-        const size_t n_q = (size_t)n_rows * (I / 4);
-        LAUNCH(s, swiglu_kernel<T>, (unsigned)((n_q + 255) / 256), 256, 0, acc, I, (T*)s->act_i, (size_t)I, n_rows, s->row_pos);
+        bool fused = false;
+        RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, n_rows, &acc, (T*)s->act_i, &fused));
+        if (!fused) {
+            const size_t n_q = (size_t)n_rows * (I / 4);
+            LAUNCH(s, swiglu_kernel<T>, (unsigned)((n_q + 255) / 256), 256, 0, acc, I, (T*)s->act_i, (size_t)I, n_rows, s->row_pos,
+                   s->m->gu_interleaved ? 1 : 0);
+        }
         RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, n_rows, &out->src));
         out->resid = s->x;
         return RD_OK;

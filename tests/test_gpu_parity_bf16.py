@@ -229,3 +229,29 @@ def test_twin_long_context_batch_4_window_32():
     assert all(len(sq.window) == 21 for sq in seqs)
     print(f"near-ties {ls.near_ties} of {ls.n_drafts}, max err {ls.max_err}")
     assert _ties_ok(ls)
+
+
+@pytest.mark.parametrize("rows", [(1, 4), (4, 8), (8, 16), (16, 16)])
+def test_twin_unfused_swiglu_path_and_fused_agree(rows):
+    """The gate/up projection with the SwiGLU in its epilogue (default) and with partial sums plus a
+    separate kernel: the second is run in lock step with the oracle here (the first everywhere else),
+    and the two give the same tokens and latents within the rounding of the different summation order.
+    Row counts cover the 16-, 32-, 128- and 256-row tiles."""
+    B, W = rows
+    lens = rd_inputs.make_prompt_lengths(B, 5, 40, seed=6)
+    model, gm, sess, sm = _setup(rd_inputs.TWIN, W, 12, batch=B, cap=8, max_ctx=96, adapter_s_scale=0.25)
+    sess.set_fused_swiglu(False)
+    seqs = _prefill_both(sm, sess, rd_inputs.TWIN, lens, 2, 12)
+    ls = LockStep(sm, sess, seqs, TOL, tie_gap=TIE_GAP)
+    for _ in range(10):
+        ls.df(W, 1, 0.0)
+    assert _ties_ok(ls)
+    z_unfused = sess.debug_read(rd.RD_DBG_LATENTS, 0).copy()
+    sess2 = rd.Session(gm, batch=B, max_context=96, max_window=W, max_iters_per_pos=8, max_new_tokens=12,
+                       keep_logits=True, seed=7)
+    for b, L in enumerate(lens):
+        sess2.prefill(b, rd_inputs.make_prompt(int(L), rd_inputs.TWIN["vocab"], seed=b), 2)
+    for _ in range(10):
+        sess2.df_step(W, 1, 0.0)
+    z_fused = sess2.debug_read(rd.RD_DBG_LATENTS, 0)
+    assert z_fused.shape == z_unfused.shape and np.abs(z_fused - z_unfused).max() < 5e-2
