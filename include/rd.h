@@ -257,6 +257,12 @@ int rd_set_gemm_path(rd_session* s, int32_t path);
  * 0: ordinary stream-ordered launches.  Results are identical; for measurement and tests. */
 int rd_set_launch_chaining(rd_session* s, int32_t on);
 
+/* rd_set_attention_path -- 2 (default for RD_BF16 with head_dim 64, 96 or 128): windowed tensor-core
+ * attention with K and V brought in by TMA through a ring of barrier-guarded stages; 1: the same
+ * arithmetic with K and V brought in by cp.async, double buffered; 0: one block per (row, head).
+ * For measurement (A/B) and tests.  STATE when the model cannot take the requested path. */
+int rd_set_attention_path(rd_session* s, int32_t path);
+
 /* rd_set_fused_swiglu -- 1 (default): on the tensor-core path the gate/up projection runs on whole
  * tiles and its epilogue writes silu(gate) * up directly (no partial sums, no separate kernel);
  * 0: the projection leaves partial sums and a separate kernel applies the SwiGLU.  Same arithmetic up

@@ -18,7 +18,7 @@ EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
            "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining",
-           "rd_debug_expire_next_wait", "rd_set_fused_swiglu"]
+           "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path"]
 
 
 class RdConfig(C.Structure):
@@ -85,6 +85,7 @@ def lib():
         L.rd_set_launch_chaining.argtypes = [vp, i32]
         L.rd_debug_expire_next_wait.argtypes = [vp]
         L.rd_set_fused_swiglu.argtypes = [vp, i32]
+        L.rd_set_attention_path.argtypes = [vp, i32]
         L.rd_profile_enable.argtypes = [vp, i32]
         L.rd_profile_read.argtypes = [vp, C.POINTER(RdProfile)]
         L.rd_strerror.argtypes = [C.c_int]
@@ -236,6 +237,9 @@ class Session:
 
     def set_launch_chaining(self, on):
         _check(lib().rd_set_launch_chaining(self.handle, 1 if on else 0), "rd_set_launch_chaining")
+
+    def set_attention_path(self, path):
+        _check(lib().rd_set_attention_path(self.handle, path), "rd_set_attention_path")
 
     def set_fused_swiglu(self, on):
         _check(lib().rd_set_fused_swiglu(self.handle, 1 if on else 0), "rd_set_fused_swiglu")

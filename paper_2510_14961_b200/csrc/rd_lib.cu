@@ -272,10 +272,14 @@ struct rd_session {
     size_t acc_elems = 0;
     bool fuse_swiglu = true;       // gate/up GEMM on whole tiles with the SwiGLU in its epilogue (tensor-core path)
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
+    int att_blk = 0, att_layer = 0;   // block and layer of the attention launch being enqueued
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
     std::vector<int> grp_ctx;   // the same bound per attention group (sequence in decode, row block in prefill)
-    int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128)
+    int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128), K/V by cp.async;
+                                // 2: the same fed by TMA through an mbarrier ring (needs the tensor maps below)
+    bool att_maps_ok = false, attn_capable = false;
+    AttMaps att_maps[3];        // per block: boxes of 64 and 32 columns over the K and the V cache
     void *act_h = nullptr, *act_2h = nullptr, *act_i = nullptr, *q_t = nullptr;
     void *Kc[3] = {nullptr, nullptr, nullptr}, *Vc[3] = {nullptr, nullptr, nullptr};
     TcAct t_act_h, t_act_2h, t_act_i;
@@ -349,6 +353,9 @@ template <int D> static cudaError_t attn_configure_d() {
     set(attn_window_kernel<D, 32, 4>, AttCfg<D, 4>::SMEM);
     set(attn_window_kernel<D, 64, 4>, AttCfg<D, 4>::SMEM);
     set(attn_window_kernel<D, 64, 8>, AttCfg<D, 8>::SMEM);
+    set(attn_tma_kernel<D, 32, 4>, AttTmaCfg<D, 4>::SMEM);
+    set(attn_tma_kernel<D, 64, 4>, AttTmaCfg<D, 4>::SMEM);
+    set(attn_tma_kernel<D, 64, 8>, AttTmaCfg<D, 8>::SMEM);
     return e;
 }
 // Function attributes (shared-memory opt-in, carve-out preference) are kept per device: they are
@@ -378,6 +385,21 @@ static int configure_device_kernels(int device) {
     if (e != cudaSuccess) return cuda_fail(e, "shared-memory opt-in of the attention kernels", __LINE__);
     g_device_configured[device] = true;
     return RD_OK;
+}
+
+// 2-D bf16 tensor [rows, D] over a K or V cache, box {cols, 64 keys}: 128-byte swizzle for boxes of
+// 64 columns, 64-byte swizzle for boxes of 32; elements outside the tensor read as zero.
+static int attn_encode(CUtensorMap* map, const void* ptr, unsigned long long rows, int D, int cols) {
+    if (!g_encode_tiled) return RD_E_STATE;
+    if (((uintptr_t)ptr & 15) != 0 || (D * 2) % 16 != 0) return RD_E_INVALID_ARG;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)ATT_KT};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RD_OK : RD_E_CUDA;
 }
 
 extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp, void* cuda_stream,
@@ -486,6 +508,20 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if (e != cudaSuccess) { rc = cuda_fail(e, "session init copies", __LINE__); break; }
         if (c.dtype == RD_BF16 && (c.head_dim == 64 || c.head_dim == 96 || c.head_dim == 128)) {
             s->attn_path = 1;
+            s->attn_capable = true;
+            // TMA view of each cache: [layers * sequences * heads * max_context, head_dim], row coordinates stay below 2^31
+            bool maps_ok = tc_init_driver() == RD_OK;
+            for (int blk = 0; blk < 3 && maps_ok; blk++) {
+                const unsigned long long rows = (unsigned long long)n_layers_of(c, blk) * B * c.n_heads * sc.max_context;
+                if (rows == 0) continue;
+                if (rows + ATT_KT >= (1ull << 31)) { maps_ok = false; break; }
+                maps_ok &= attn_encode(&s->att_maps[blk].k64, s->Kc[blk], rows, c.head_dim, 64) == RD_OK;
+                maps_ok &= attn_encode(&s->att_maps[blk].v64, s->Vc[blk], rows, c.head_dim, 64) == RD_OK;
+                maps_ok &= attn_encode(&s->att_maps[blk].k32, s->Kc[blk], rows, c.head_dim, 32) == RD_OK;
+                maps_ok &= attn_encode(&s->att_maps[blk].v32, s->Vc[blk], rows, c.head_dim, 32) == RD_OK;
+            }
+            s->att_maps_ok = maps_ok;
+            if (maps_ok) s->attn_path = 2;
         }
         if (m->tc_ok) {
             // scratch for the partial sums: the largest need over the model's GEMM shapes and over
@@ -525,6 +561,14 @@ extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
     if (!s || path < 0 || path > 2) return RD_E_INVALID_ARG;
     if (path >= 1 && !(s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
     s->gemm_path = path;
+    return RD_OK;
+}
+
+extern "C" int rd_set_attention_path(rd_session* s, int32_t path) {
+    if (!s || path < 0 || path > 2) return RD_E_INVALID_ARG;
+    if (path >= 1 && !s->attn_capable) return RD_E_STATE;             // no tensor-core attention for this model
+    if (path == 2 && !s->att_maps_ok) return RD_E_STATE;
+    s->attn_path = path;
     return RD_OK;
 }
 
@@ -653,6 +697,14 @@ template <typename T> struct Eng {
             for (int g = 0; g < groups; g++) order.idx[g] = (unsigned char)ids[g];
             order.n = groups;
         }
+        if (s->attn_path == 2) {
+            // K/V through the TMA ring; Kc points at this layer inside block s->att_blk
+            const int row_base = s->att_layer * s->sc.batch * c.n_heads * s->sc.max_context;
+            LAUNCH_CLUSTER(s, (attn_tma_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttTmaCfg<D, NW>::SMEM), ns,
+                           s->att_maps[s->att_blk], order, (const bf16*)s->q_t, s->row_pos, s->row_seq, s->grp_rows, n_rows, row_base,
+                           c.n_heads, s->sc.max_context, c.hidden, scale_log2, (bf16*)s->act_h, s->status);
+            return RD_OK;
+        }
         LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttCfg<D, NW>::SMEM), ns, order, (const bf16*)s->q_t,
                        s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
                        (bf16*)s->act_h);
@@ -695,7 +747,8 @@ template <typename T> struct Eng {
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
         if constexpr (sizeof(T) == 2) {
-            if (s->attn_path == 1 && s->grp_rows >= 1 && s->grp_rows <= ATT_QMAX) {
+            if (s->attn_path >= 1 && s->grp_rows >= 1 && s->grp_rows <= ATT_QMAX) {
+                s->att_blk = blk; s->att_layer = l;
                 RD_TRY(attn_windowed(s, Kc, Vc, n_rows));
                 windowed = true;
             }

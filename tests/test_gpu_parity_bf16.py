@@ -255,3 +255,28 @@ def test_twin_unfused_swiglu_path_and_fused_agree(rows):
         sess2.df_step(W, 1, 0.0)
     z_fused = sess2.debug_read(rd.RD_DBG_LATENTS, 0)
     assert z_fused.shape == z_unfused.shape and np.abs(z_fused - z_unfused).max() < 5e-2
+
+
+@pytest.mark.parametrize("W,batch,L", [(8, 2, 700), (64, 1, 300), (128, 1, 90)])
+def test_attention_paths_agree_bit_for_bit(W, batch, L):
+    """K and V through the TMA ring (default, run in lock step with the oracle everywhere else) and
+    through cp.async feed the same tensor-core arithmetic in the same order: tokens, latents and cache
+    rows must be identical.  Covers the half-tile warps (groups of up to 32 rows), the four-warp and the
+    eight-warp groups, several key tiles and splits."""
+    shape = rd_inputs.TWIN
+    w = rd_inputs.make_weights(**rd_inputs.shape_args(shape), seed=21, bf16=True, adapter_s_scale=0.25)
+    gm = gpu_model(shape, w, bf16=True)
+    outs = []
+    for path in (2, 1):
+        sess = rd.Session(gm, batch=batch, max_context=L + 160, max_window=W, max_new_tokens=W + 12, seed=13, temperature=0.7)
+        sess.set_attention_path(path)
+        for b in range(batch):
+            sess.prefill(b, rd_inputs.make_prompt(L - 37 * b, shape["vocab"], seed=30 + b), 2)
+        for _ in range(W + 6):
+            sess.df_step(W, 1, 0.0)
+        outs.append([sess.tokens(b).copy() for b in range(batch)] + [sess.debug_read(rd.RD_DBG_LATENTS, 0).copy(),
+                    sess.read_kv(1, 3, 0, 0, 0, L + 4), sess.read_kv(2, 1, 1, batch - 1, 0, L - 37 * (batch - 1) + 4)])
+        sess.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+    gm.close()
