@@ -85,6 +85,15 @@ typedef struct {
                                   cumulative probability under softmax(logits / temperature) reaches
                                   top_p (equal logits at the cut stay together), renormalised;
                                   0 or 1 = off.  Needs vocab <= 65536 (else INVALID_ARG)          */
+    int32_t latent_slots;      /* Appendix, "Larger Batch Sizes": number of slots for in-flight hidden
+                                  states shared by all sequences of the session (the paper's "occupancy
+                                  multiplier" times max_window).  0 or batch * max_window: every
+                                  sequence owns max_window slots.  Fewer: slots are handed out from a
+                                  pool as positions enter a wavefront and returned when they are
+                                  committed; a sequence that finds the pool empty does not append a
+                                  position that step (it stalls as at a full wavefront) and goes on
+                                  when a slot is returned.  Slots go to sequences in index order.
+                                  Needs batch <= 1024 (CAPACITY)                                   */
 } rd_session_config;
 
 typedef struct {

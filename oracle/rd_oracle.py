@@ -363,10 +363,11 @@ class Sampler:
     def _sample(self, logits, seq_id, token_pos):
         return sample_token(logits, self.temperature, self.seed, seq_id, token_pos, self.top_p)
 
-    def prefill(self, seq_id, prompt, r, max_new):
+    def prefill(self, seq_id, prompt, r, max_new, first_row=True):
         """Section 3.3: the prompt's positions 0..L-2 run P, r simultaneous passes of R and the
         coda layers (to fill its cache).  Position L-1 becomes the first in-flight position with
-        a fresh state (the initialisation steps of Algorithm 1)."""
+        a fresh state (the initialisation steps of Algorithm 1); first_row=False leaves the
+        wavefront empty (no slot free for its hidden state yet, see df_step's may_append)."""
         prompt = np.asarray(prompt, dtype=np.int64)
         L = len(prompt)
         assert L >= 1 and L + max_new <= self.m.max_ctx
@@ -380,7 +381,7 @@ class Sampler:
             for _ in range(r):
                 s = self.m.core(e, s, pos, sq.caches)
             self.m.coda(s, pos, sq.caches, head=False)
-        sq.window = [Row(L - 1, self._init(seq_id, L - 1))]
+        sq.window = [Row(L - 1, self._init(seq_id, L - 1))] if first_row else []
         sq.done = max_new <= 0
         if sq.done:
             sq.window = []
@@ -408,13 +409,26 @@ class Sampler:
             sq.window = [Row(row.pos + 1, self._init(sq.seq_id, row.pos + 1))]
         return info
 
-    def df_step(self, sq: Sequence, window, inner_iters, exit_threshold):
+    def df_step(self, sq: Sequence, window, inner_iters, exit_threshold, may_append=True):
         """One step of the diffusion-forcing sampler (Algorithm 1 when exit_threshold <= 0,
-        Algorithm 2 otherwise).  Returns what the step computed, for inspection."""
+        Algorithm 2 otherwise).  Returns what the step computed, for inspection.
+
+        may_append=False: the engine has no slot for a further hidden state this step (Appendix,
+        "Larger Batch Sizes": a bounded number of slots shared by the sequences), so the wavefront is
+        not extended, exactly as when it is full (Section 3.5); nothing else changes.  A sequence may
+        then hold no in-flight position at all: the step computes nothing for it and only appends."""
         if sq.done:
             return None
         rows = sq.window
-        assert 1 <= len(rows) <= window
+        assert len(rows) <= window
+        if not rows:
+            info = {"pos": np.zeros(0, dtype=np.int64), "z": np.zeros((0, self.m.cfg.hidden), dtype=self.m.dtype),
+                    "logits": np.zeros((0, self.m.cfg.vocab), dtype=self.m.dtype), "drafts": np.zeros(0, dtype=np.int64),
+                    "delta": np.zeros(0, dtype=np.float32), "n_commit": 0}
+            if may_append:
+                nxt = sq.n_committed - 1
+                sq.window.append(Row(nxt, self._init(sq.seq_id, nxt)))
+            return info
         pos = np.array([r_.pos for r_ in rows])
         # e <- P(y_current): the oldest row reads the last committed token, the others the
         # drafts of the previous step.
@@ -466,7 +480,7 @@ class Sampler:
         last_row_pos = sq.n_prompt + sq.max_new - 2       # its draft is the last token wanted
         if sq.n_committed - sq.n_prompt >= sq.max_new:
             sq.done, sq.window = True, []
-        elif len(sq.window) < window:
+        elif len(sq.window) < window and may_append:
             nxt = sq.n_committed - 1 + len(sq.window)
             if nxt <= last_row_pos:
                 sq.window.append(Row(nxt, self._init(sq.seq_id, nxt)))

@@ -31,7 +31,7 @@ class RdSessionConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("batch", "max_context", "max_window", "max_iters_per_pos",
                                          "max_new_tokens", "keep_logits")] + \
                [("temperature", C.c_float), ("seed", C.c_uint64), ("eta", C.c_float), ("beta", C.c_float),
-                ("top_p", C.c_float)]
+                ("top_p", C.c_float), ("latent_slots", C.c_int32)]
 
 
 class RdStats(C.Structure):
@@ -146,10 +146,10 @@ class Session:
 
     def __init__(self, model: Model, batch=1, max_context=1024, max_window=1, max_iters_per_pos=64,
                  max_new_tokens=64, keep_logits=False, temperature=0.0, seed=0, stream=None, eta=0.0, beta=0.0,
-                 top_p=0.0):
+                 top_p=0.0, latent_slots=0):
         self.model = model
         self.sc = RdSessionConfig(batch, max_context, max_window, max_iters_per_pos, max_new_tokens,
-                                  1 if keep_logits else 0, temperature, seed, eta, beta, top_p)
+                                  1 if keep_logits else 0, temperature, seed, eta, beta, top_p, latent_slots)
         self.handle = C.c_void_p()
         _check(lib().rd_session_create(model.handle, C.byref(self.sc), C.c_void_p(stream or 0),
                                        C.byref(self.handle)), "rd_session_create")

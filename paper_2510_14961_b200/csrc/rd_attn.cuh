@@ -58,7 +58,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int D, int NW> struct AttCfg {
     static constexpr int LD = D + 8;    // padded row (elements): ldmatrix rows fall in distinct banks
     static constexpr int QMAX = 16 * NW;   // queries a CTA of NW warps holds
-    static constexpr int SMEM = (QMAX * LD + 4 * ATT_KT * LD) * 2 + QMAX * 4;
+    static constexpr int SMEM = (QMAX * LD + 4 * ATT_KT * LD) * 2 + 2 * QMAX * 4;   // Q, K/V double buffer, positions, row indices
 };
 
 // Grid (splits, heads, groups), clusters of `splits` blocks along x.  out: [rows, hidden] bf16.
@@ -77,7 +77,7 @@ struct GroupOrder {
 template <int D, int KW, int NW>
 __global__ void __launch_bounds__(32 * NW)
 attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t, const int* __restrict__ row_pos,
-                   const int* __restrict__ row_seq, int rows_per_group, int n_rows,
+                   const int* __restrict__ row_seq, const int* __restrict__ grp_index, int rows_per_group, int n_rows,
                    const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc, size_t seq_stride,
                    size_t head_stride, int hidden, float scale_log2, __nv_bfloat16* __restrict__ out) {
     constexpr int LD = AttCfg<D, NW>::LD;
@@ -90,16 +90,20 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     __nv_bfloat16* Ks = Qs + QMAX * LD;                   // [2][KT][LD]
     __nv_bfloat16* Vs = Ks + 2 * ATT_KT * LD;             // [2][KT][LD]
     int* pos_s = (int*)(Vs + 2 * ATT_KT * LD);
+    int* ridx_s = pos_s + QMAX;
 
     pdl_enter();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sp = blockIdx.x, n_splits = gridDim.x, hd = blockIdx.y;
-    const int r0 = (order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z) * rows_per_group;
-    const int nq = min(rows_per_group, n_rows - r0);
+    const int grp = order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z;
+    const int r0 = grp * rows_per_group;
+    // rows of the group: consecutive rows r0 .. of the row table, or (pooled slots) the rows grp_index lists
+    const int nq = grp_index ? rows_per_group : min(rows_per_group, n_rows - r0);
     // positions of the group's rows; kv_len = 1 + the largest of them
     __shared__ int warp_max[NW];
-    const int my_pos = (tid < QMAX && tid < nq) ? row_pos[r0 + tid] : -1;
-    if (tid < QMAX) pos_s[tid] = my_pos;
+    const int my_row = (tid < QMAX && tid < nq) ? (grp_index ? grp_index[r0 + tid] : r0 + tid) : -1;
+    const int my_pos = my_row >= 0 ? row_pos[my_row] : -1;
+    if (tid < QMAX) { pos_s[tid] = my_pos; ridx_s[tid] = my_row; }
     const int wmax = __reduce_max_sync(0xffffffffu, my_pos);
     if (lane == 0) warp_max[warp] = wmax;
     __syncthreads();
@@ -108,7 +112,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     for (int w = 0; w < NW; w++) kv_len = max(kv_len, warp_max[w] + 1);
     const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
     const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
-    const int seq = row_seq[r0];
+    const int seq = grp_index ? grp : row_seq[r0];          // pooled slots: group = sequence
     // cache layout [sequence][head][position][D]: this head's keys are one contiguous stream
     const __nv_bfloat16* kbase = Kc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
     const __nv_bfloat16* vbase = Vc + (size_t)seq * seq_stride + (size_t)hd * head_stride;
@@ -116,7 +120,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     for (int c = tid; c < QMAX * CH; c += NT) {
         const int r = c / CH, ch = c % CH;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)(r0 + r) * hidden + hd * D + ch * 8);
+        if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)ridx_s[r] * hidden + hd * D + ch * 8);
         *reinterpret_cast<uint4*>(Qs + r * LD + ch * 8) = v;
     }
     auto load_tile = [&](int t, int buf) {
@@ -280,7 +284,8 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
     const int mine = nq > sp ? (nq - sp + n_splits - 1) / n_splits : 0;
     for (int item = tid; item < mine * Q4; item += NT) {
         const int q = sp + (item / Q4) * n_splits, e = (item % Q4) * 4;
-        __nv_bfloat16* dst = out + (size_t)(r0 + q) * hidden + hd * D + e;
+        if (ridx_s[q] < 0) continue;                          // no row behind this entry of the group
+        __nv_bfloat16* dst = out + (size_t)ridx_s[q] * hidden + hd * D + e;
         float2 ml[ATT_MAX_SPLITS];
         float4 po[ATT_MAX_SPLITS];
 #pragma unroll
@@ -387,7 +392,7 @@ template <int D, int NW> struct AttTmaCfg {
     static constexpr int RING = STAGES * STAGE_BYTES;
     static constexpr int Q_BYTES = QMAX * LD * 2;
     // ring (1024-aligned) | Q | positions | barriers
-    static constexpr int SMEM = 1024 + RING + Q_BYTES + QMAX * 4 + 2 * STAGES * 8 + 16;
+    static constexpr int SMEM = 1024 + RING + Q_BYTES + 2 * QMAX * 4 + 2 * STAGES * 8 + 16;
     static_assert(QMAX * D * 4 + QMAX * 8 + 64 * (D / 2 + 4) * 4 <= RING, "merge area fits in the ring");
 };
 
@@ -400,8 +405,8 @@ struct AttMaps {
 template <int D, int KW, int NW>
 __global__ void __launch_bounds__(32 * NW, NW == 4 ? 3 : 1)
 attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, const __nv_bfloat16* __restrict__ q_t,
-                const int* __restrict__ row_pos, const int* __restrict__ row_seq, int rows_per_group, int n_rows,
-                int row_base, int n_heads, int max_context, int hidden, float scale_log2,
+                const int* __restrict__ row_pos, const int* __restrict__ row_seq, const int* __restrict__ grp_index,
+                int rows_per_group, int n_rows, int row_base, int n_heads, int max_context, int hidden, float scale_log2,
                 __nv_bfloat16* __restrict__ out, int* __restrict__ status) {
     using C = AttTmaCfg<D, NW>;
     using T = AttTile<D>;
@@ -411,7 +416,8 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     uint8_t* ring = (uint8_t*)(((uintptr_t)att_raw + 1023) & ~(uintptr_t)1023);
     __nv_bfloat16* Qs = (__nv_bfloat16*)(ring + C::RING);
     int* pos_s = (int*)(ring + C::RING + C::Q_BYTES);
-    uint64_t* full = (uint64_t*)(pos_s + QMAX);
+    int* ridx_s = pos_s + QMAX;
+    uint64_t* full = (uint64_t*)(ridx_s + QMAX);
     uint64_t* empty = full + S;
     __shared__ int warp_max[NW];
     __shared__ int abort_s;
@@ -432,10 +438,12 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     }
     pdl_enter();
     const int sp = blockIdx.x, n_splits = gridDim.x, hd = blockIdx.y;
-    const int r0 = (order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z) * rows_per_group;
-    const int nq = min(rows_per_group, n_rows - r0);
-    const int my_pos = (tid < QMAX && tid < nq) ? row_pos[r0 + tid] : -1;
-    if (tid < QMAX) pos_s[tid] = my_pos;
+    const int grp = order.n ? (int)order.idx[blockIdx.z] : (int)blockIdx.z;
+    const int r0 = grp * rows_per_group;
+    const int nq = grp_index ? rows_per_group : min(rows_per_group, n_rows - r0);
+    const int my_row = (tid < QMAX && tid < nq) ? (grp_index ? grp_index[r0 + tid] : r0 + tid) : -1;
+    const int my_pos = my_row >= 0 ? row_pos[my_row] : -1;
+    if (tid < QMAX) { pos_s[tid] = my_pos; ridx_s[tid] = my_row; }
     const int wmax = __reduce_max_sync(0xffffffffu, my_pos);
     if (lane == 0) warp_max[warp] = wmax;
     __syncthreads();                                       // barriers initialised, positions visible
@@ -445,7 +453,7 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     const int n_tiles = (kv_len + ATT_KT - 1) / ATT_KT;
     const int t0 = (int)((long long)sp * n_tiles / n_splits), t1 = (int)((long long)(sp + 1) * n_tiles / n_splits);
     const int nt = t1 - t0;
-    const int seq = row_seq[r0];
+    const int seq = grp_index ? grp : row_seq[r0];          // pooled slots: group = sequence
     const int head_row0 = row_base + (seq * n_heads + hd) * max_context;   // row of this head's position 0
 
     auto issue = [&](int it) {                              // thread 0: tile t0 + it into stage it % S
@@ -472,7 +480,7 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     for (int c = tid; c < QMAX * CH; c += NT) {
         const int r = c / CH, ch = c % CH;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)(r0 + r) * hidden + hd * D + ch * 8);
+        if (r < nq && pos_s[r] >= 0) v = *reinterpret_cast<const uint4*>(q_t + (size_t)ridx_s[r] * hidden + hd * D + ch * 8);
         *reinterpret_cast<uint4*>(Qs + r * LD + ch * 8) = v;
     }
     const int qblk = KW == 64 ? warp : (warp & 1);        // block of 16 queries this warp takes
@@ -635,7 +643,8 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     const int mine = nq > sp ? (nq - sp + n_splits - 1) / n_splits : 0;
     for (int item = tid; item < mine * Q4; item += NT) {
         const int q = sp + (item / Q4) * n_splits, e = (item % Q4) * 4;
-        __nv_bfloat16* dst = out + (size_t)(r0 + q) * hidden + hd * D + e;
+        if (ridx_s[q] < 0) continue;                          // no row behind this entry of the group
+        __nv_bfloat16* dst = out + (size_t)ridx_s[q] * hidden + hd * D + e;
         float2 ml[ATT_MAX_SPLITS];
         float4 po[ATT_MAX_SPLITS];
 #pragma unroll

@@ -995,6 +995,144 @@ __global__ void seq_start_kernel(SeqState st, int seq, int L, int slot, int is_d
     st.row_iters[slot] = 0;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Pooled latent slots (Appendix, "Larger Batch Sizes": a number of slots for hidden states, an
+// occupancy multiple of the maximum wavefront, shared by the sequences; a slot need not belong to a
+// contiguous run of positions).  ring[b * Wmax + (p mod Wmax)] names the slot that holds in-flight
+// position p of sequence b (-1: none); free_list[0 .. *free_top) are the unused slots.
+// ---------------------------------------------------------------------------------------------
+struct SlotPool {
+    int* ring;        // [B * Wmax]
+    int* free_list;   // [n_slots]
+    int* free_top;    // [1]
+};
+
+// Row tables of a decode step from the ring: row = slot.  One block.  grp_index[b * Wmax + i] = slot of
+// the i-th in-flight position of sequence b (-1 beyond its wavefront): the attention kernel's groups.
+__global__ void plan_rows_pool_kernel(const int* __restrict__ n_committed, const int* __restrict__ win_len,
+                                      const int* __restrict__ done, int B, int Wmax, int n_slots, SlotPool pool,
+                                      int* __restrict__ row_pos, int* __restrict__ row_seq, int* __restrict__ grp_index,
+                                      int* __restrict__ step_first, int* __restrict__ step_n) {
+    pdl_enter();
+    for (int s = threadIdx.x; s < n_slots; s += blockDim.x) { row_pos[s] = -1; row_seq[s] = 0; }
+    __syncthreads();
+    for (int e = threadIdx.x; e < B * Wmax; e += blockDim.x) {
+        const int b = e / Wmax, i = e % Wmax;
+        const int f = n_committed[b] - 1;
+        const int w = done[b] ? 0 : win_len[b];
+        int slot = -1;
+        if (i < w) {
+            slot = pool.ring[b * Wmax + (f + i) % Wmax];
+            row_pos[slot] = f + i;
+            row_seq[slot] = b;
+        }
+        grp_index[e] = slot;
+        if (i == 0) { step_first[b] = f; step_n[b] = w; }
+    }
+}
+
+// advance_kernel for pooled slots.  One block, one thread per sequence (B <= blockDim.x) for the
+// freeze / commit decisions; then thread 0 returns the slots of the rows that left (sequences in
+// index order) and hands free slots to the sequences that want to append a row (index order again):
+// a sequence that finds no free slot does not append this step (it stalls, like a full wavefront).
+__global__ void advance_pool_kernel(SeqState st, const float* __restrict__ delta, int B, int Wmax, int window,
+                                    int inner_iters, float exit_threshold, int cap, int max_new, int layer_passes,
+                                    SlotPool pool) {
+    extern __shared__ int sh[];                  // [B] rows dropped, [B] their first position, [B] position to append or -1
+    int* dropped = sh;
+    int* first = sh + B;
+    int* want = sh + 2 * B;
+    pdl_enter();
+    const int b = threadIdx.x;
+    if (b < B) { dropped[b] = 0; first[b] = 0; want[b] = -1; }
+    if (b < B && !st.done[b]) {
+        const int f = st.n_committed[b] - 1;
+        int w = st.win_len[b];
+        int k = 0;
+        bool open = true;
+        for (int i = 0; i < w; i++) {
+            const int s = pool.ring[b * Wmax + (f + i) % Wmax];
+            const int steps = ++st.row_steps[s];
+            const int iters = (st.row_iters[s] += inner_iters);
+            const bool fin = exit_threshold <= 0.f ? steps >= window : (delta[s] < exit_threshold || iters >= cap);
+            if (open && fin) k++; else open = false;
+        }
+        atomicAdd(&st.counters[0], (unsigned long long)w);
+        atomicAdd(&st.counters[1], (unsigned long long)w * inner_iters);
+        atomicAdd(&st.counters[2], (unsigned long long)w);
+        if (w > 0) {
+            atomicAdd(&st.counters[4], (unsigned long long)(f + w) * layer_passes);
+            atomicAdd(&st.counters[5], ((unsigned long long)w * (f + 1) + (unsigned long long)w * (w - 1) / 2) * layer_passes);
+        }
+        int nc = st.n_committed[b];
+        const int np = st.n_prompt[b];
+        k = min(k, max_new - (nc - np));
+        nc += k;
+        first[b] = f;                            // the rows that leave are the oldest ones: positions f, f + 1, ...
+        atomicAdd(&st.counters[3], (unsigned long long)k);
+        atomicAdd(&st.counters[RD_HIST_AT + min(k, RD_HIST_BINS - 1)], 1ull);
+        if (nc - np >= max_new) {
+            st.done[b] = 1;
+            dropped[b] = w;                      // everything this sequence held
+            w = 0;
+        } else {
+            dropped[b] = k;
+            w -= k;
+            if (w < window) {
+                const int nxt = nc - 1 + w;
+                if (nxt <= np + max_new - 2) want[b] = nxt;
+            }
+        }
+        st.n_committed[b] = nc;
+        st.win_len[b] = w;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int top = *pool.free_top;
+        for (int q = 0; q < B; q++)
+            for (int i = 0; i < dropped[q]; i++) {
+                const int e = q * Wmax + (first[q] + i) % Wmax;
+                pool.free_list[top++] = pool.ring[e];
+                pool.ring[e] = -1;
+            }
+        for (int q = 0; q < B; q++) {
+            if (want[q] < 0 || top == 0) continue;
+            const int s = pool.free_list[--top];
+            pool.ring[q * Wmax + want[q] % Wmax] = s;
+            st.row_steps[s] = 0;
+            st.row_iters[s] = 0;
+            st.win_len[q] += 1;
+        }
+        *pool.free_top = top;
+    }
+}
+
+// seq_start_kernel for pooled slots: a restarted sequence first returns what it held, then takes one
+// slot for position L-1 if one is free (otherwise it starts with an empty wavefront and gets its
+// first row from advance_pool_kernel as soon as a slot frees up).
+__global__ void seq_start_pool_kernel(SeqState st, int seq, int L, int Wmax, int is_done, SlotPool pool) {
+    pdl_enter();
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    int top = *pool.free_top;
+    for (int j = 0; j < Wmax; j++) {
+        const int s = pool.ring[seq * Wmax + j];
+        if (s >= 0) { pool.free_list[top++] = s; pool.ring[seq * Wmax + j] = -1; }
+    }
+    int w = 0;
+    if (!is_done && top > 0) {
+        const int s = pool.free_list[--top];
+        pool.ring[seq * Wmax + (L - 1) % Wmax] = s;
+        st.row_steps[s] = 0;
+        st.row_iters[s] = 0;
+        w = 1;
+    }
+    *pool.free_top = top;
+    st.n_prompt[seq] = L;
+    st.n_committed[seq] = L;
+    st.win_len[seq] = w;
+    st.done[seq] = is_done;
+}
+
 // float32 -> T copy (weight upload path; bf16 rounds to nearest even once).
 template <typename T>
 __global__ void convert_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {

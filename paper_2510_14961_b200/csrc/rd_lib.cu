@@ -272,6 +272,11 @@ struct rd_session {
     size_t acc_elems = 0;
     bool fuse_swiglu = true;       // gate/up GEMM on whole tiles with the SwiGLU in its epilogue (tensor-core path)
     bool chained = true;           // launch the step's kernels as a programmatic-dependent-launch chain
+    bool pooled = false;        // latent slots drawn from a pool smaller than batch * max_window
+    SlotPool pool = {nullptr, nullptr, nullptr};
+    int* grp_index = nullptr;   // pooled: per sequence, the slots of its in-flight rows (attention groups)
+    const int* att_index = nullptr;   // grp_index during a pooled decode step, null otherwise
+    int att_groups = 0;         // attention groups of the pass when they are not n_rows / grp_rows
     int att_blk = 0, att_layer = 0;   // block and layer of the attention launch being enqueued
     int grp_rows = 0;           // rows per attention query group in the current pass
     int ctx_max = 0;            // host-side upper bound of the longest context in the current pass
@@ -413,6 +418,9 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     // the top-p kernel keeps a row's logits in the registers of one cluster
     if (sc.temperature > 0.f && sc.top_p > 0.f && sc.top_p < 1.f && m->cfg.vocab > NUC_MAX_VOCAB) return RD_E_INVALID_ARG;
     if ((long long)sc.batch * sc.max_window > 4096) return RD_E_CAPACITY;
+    if (sc.latent_slots < 0 || (long long)sc.latent_slots > (long long)sc.batch * sc.max_window) return RD_E_INVALID_ARG;
+    const bool pooled = sc.latent_slots > 0 && sc.latent_slots < sc.batch * sc.max_window;
+    if (pooled && sc.batch > 1024) return RD_E_CAPACITY;        // one thread per sequence in the pool's bookkeeping kernel
     {
         int dev = -1;
         CU(cudaGetDevice(&dev));
@@ -427,7 +435,8 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
     memset(&s->stats, 0, sizeof s->stats);
     const rd_config& c = m->cfg;
     const size_t h = c.hidden, I = c.mlp_inner, V = c.vocab, es = m->esz;
-    s->n_slots = sc.batch * sc.max_window;
+    s->pooled = pooled;
+    s->n_slots = pooled ? sc.latent_slots : sc.batch * sc.max_window;
     s->R = std::max(s->n_slots, 512);   // prefill chunk: rows that share one pass over the weights
     s->R = (s->R + 15) / 16 * 16;
     s->tok_stride = sc.max_context + 1;
@@ -447,6 +456,20 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
         if ((rc = s->mem.get(&s->row_seq, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->draft, R * sizeof(int)))) break;
         if ((rc = s->mem.get(&s->counters, RD_COUNTERS * sizeof(unsigned long long)))) break;
+        if (pooled) {
+            const size_t ring_n = B * sc.max_window;
+            if ((rc = s->mem.get(&s->pool.ring, ring_n * sizeof(int)))) break;
+            if ((rc = s->mem.get(&s->pool.free_list, (size_t)s->n_slots * sizeof(int)))) break;
+            if ((rc = s->mem.get(&s->pool.free_top, sizeof(int)))) break;
+            if ((rc = s->mem.get(&s->grp_index, ring_n * sizeof(int)))) break;
+            std::vector<int> minus(ring_n, -1), fl(s->n_slots);
+            for (int i = 0; i < s->n_slots; i++) fl[i] = s->n_slots - 1 - i;      // slot 0 is handed out first
+            const int top = s->n_slots;
+            cudaError_t ep = cudaMemcpy(s->pool.ring, minus.data(), ring_n * sizeof(int), cudaMemcpyHostToDevice);
+            if (ep == cudaSuccess) ep = cudaMemcpy(s->pool.free_list, fl.data(), fl.size() * sizeof(int), cudaMemcpyHostToDevice);
+            if (ep == cudaSuccess) ep = cudaMemcpy(s->pool.free_top, &top, sizeof(int), cudaMemcpyHostToDevice);
+            if (ep != cudaSuccess) { rc = cuda_fail(ep, "slot pool init", __LINE__); break; }
+        }
         // what the host polls sits in one block (status word, |y_frozen| and done flag per sequence)
         // so that one copy into a pinned mirror brings all of it
         s->poll_ints = 4 + 2 * B;
@@ -681,7 +704,7 @@ template <typename T> struct Eng {
     template <int D, int KW, int NW>
     static int attn_windowed_d(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
         const rd_config& c = s->m->cfg;
-        const int groups = (n_rows + s->grp_rows - 1) / s->grp_rows;
+        const int groups = s->att_groups > 0 ? s->att_groups : (n_rows + s->grp_rows - 1) / s->grp_rows;
         const int tiles = std::max(1, (s->ctx_max + ATT_KT - 1) / ATT_KT);
         // enough (group, head, split) blocks for two per SM; a split never gets less than one tile
         int ns = (2 * s->m->n_sms + groups * c.n_heads - 1) / (groups * c.n_heads);
@@ -701,12 +724,12 @@ template <typename T> struct Eng {
             // K/V through the TMA ring; Kc points at this layer inside block s->att_blk
             const int row_base = s->att_layer * s->sc.batch * c.n_heads * s->sc.max_context;
             LAUNCH_CLUSTER(s, (attn_tma_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttTmaCfg<D, NW>::SMEM), ns,
-                           s->att_maps[s->att_blk], order, (const bf16*)s->q_t, s->row_pos, s->row_seq, s->grp_rows, n_rows, row_base,
+                           s->att_maps[s->att_blk], order, (const bf16*)s->q_t, s->row_pos, s->row_seq, s->att_index, s->grp_rows, n_rows, row_base,
                            c.n_heads, s->sc.max_context, c.hidden, scale_log2, (bf16*)s->act_h, s->status);
             return RD_OK;
         }
         LAUNCH_CLUSTER(s, (attn_window_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttCfg<D, NW>::SMEM), ns, order, (const bf16*)s->q_t,
-                       s->row_pos, s->row_seq, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
+                       s->row_pos, s->row_seq, s->att_index, s->grp_rows, n_rows, Kc, Vc, s->seq_stride, s->head_stride, c.hidden, scale_log2,
                        (bf16*)s->act_h);
         return RD_OK;
     }
@@ -864,8 +887,17 @@ template <typename T> struct Eng {
                 s->ctx_max = std::max(s->ctx_max, ctx);
                 s->grp_ctx[b] = ctx;
             }
-        LAUNCH(s, plan_rows_kernel, (n + 127) / 128, 128, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window,
-               s->row_pos, s->row_seq, s->step_first, s->step_n);
+        s->att_index = nullptr;
+        s->att_groups = 0;
+        if (s->pooled) {
+            LAUNCH(s, plan_rows_pool_kernel, 1, 1024, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window, n, s->pool,
+                   s->row_pos, s->row_seq, s->grp_index, s->step_first, s->step_n);
+            s->att_index = s->grp_index;
+            s->att_groups = B;
+        } else {
+            LAUNCH(s, plan_rows_kernel, (n + 127) / 128, 128, 0, s->n_committed, s->win_len, s->done, B, s->sc.max_window,
+                   s->row_pos, s->row_seq, s->step_first, s->step_n);
+        }
         // s_0 for the rows appended by the previous step, and the snapshot z_prev <- z
         // (stabilisers of Section 3.4 apply to sampler steps, not to the sequential decoder)
         const float eta = stabilise ? s->sc.eta : 0.f, beta = stabilise ? s->sc.beta : 0.f;
@@ -877,8 +909,15 @@ template <typename T> struct Eng {
         RD_TRY(coda(s, s->z, n, true));
         LAUNCH(s, delta_kernel, n, DELTA_THREADS, 0, s->z, s->z_prev, h, s->row_pos, s->delta);
         SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
-        LAUNCH(s, advance_kernel, (B + 63) / 64, 64, 0, st, s->delta, B, s->sc.max_window, window, inner, eps,
-               s->sc.max_iters_per_pos, s->sc.max_new_tokens, c.n_prelude + c.n_coda + inner * c.n_core);
+        if (s->pooled) {
+            LAUNCH(s, advance_pool_kernel, 1, (B + 31) / 32 * 32, 3 * B * sizeof(int), st, s->delta, B, s->sc.max_window, window, inner, eps,
+                   s->sc.max_iters_per_pos, s->sc.max_new_tokens, c.n_prelude + c.n_coda + inner * c.n_core, s->pool);
+        } else {
+            LAUNCH(s, advance_kernel, (B + 63) / 64, 64, 0, st, s->delta, B, s->sc.max_window, window, inner, eps,
+                   s->sc.max_iters_per_pos, s->sc.max_new_tokens, c.n_prelude + c.n_coda + inner * c.n_core);
+        }
+        s->att_index = nullptr;
+        s->att_groups = 0;
         // every weight matrix is streamed once per pass: prelude, coda and head once, core and adapter `inner` times
         const uint64_t per_layer = 4ull * h * h + 3ull * h * c.mlp_inner;
         s->stats.weight_bytes += ((uint64_t)(c.n_prelude + c.n_coda) * per_layer + (uint64_t)c.vocab * h +
@@ -895,6 +934,8 @@ template <typename T> struct Eng {
             for (int c0 = 0; c0 < n; c0 += s->R) {
                 const int nr = std::min(s->R, n - c0);
                 s->grp_rows = ATT_QMAX;
+                s->att_index = nullptr;
+                s->att_groups = 0;
                 s->ctx_max = c0 + nr;
                 s->ctx_total = c0 + nr;
                 s->grp_ctx.clear();
@@ -931,6 +972,10 @@ template <typename T> struct Eng {
         if (n > 0) RD_TRY(prefill_passes(s, seq, n, r, s->pf_e, s->pf_s));
         // sequence state: |y_frozen| = L, one fresh in-flight row at position L-1
         SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
+        if (s->pooled) {
+            LAUNCH(s, seq_start_pool_kernel, 1, 32, 0, st, seq, L, s->sc.max_window, s->sc.max_new_tokens <= 0 ? 1 : 0, s->pool);
+            return RD_OK;
+        }
         const int slot = seq * s->sc.max_window + (L - 1) % s->sc.max_window;
         LAUNCH(s, seq_start_kernel, 1, 32, 0, st, seq, L, slot, s->sc.max_new_tokens <= 0 ? 1 : 0);
         return RD_OK;
@@ -1045,8 +1090,18 @@ extern "C" int rd_debug_read(rd_session* s, int32_t what, int32_t seq, void* dst
         default: return RD_E_INVALID_ARG;
     }
     if (bytes < row_bytes * n) return RD_E_INVALID_ARG;
+    // pooled slots: the slots of the rows the last step processed, oldest first, as that step's row plan listed them
+    std::vector<int> plan;
+    if (s->pooled) {
+        plan.resize(s->sc.max_window);
+        CU(cudaMemcpy(plan.data(), s->grp_index + (size_t)seq * s->sc.max_window, plan.size() * sizeof(int), cudaMemcpyDeviceToHost));
+    }
     for (int i = 0; i < n; i++) {
-        const int slot = seq * s->sc.max_window + (f + i) % s->sc.max_window;
+        int slot = seq * s->sc.max_window + (f + i) % s->sc.max_window;
+        if (s->pooled) {
+            slot = plan[i];
+            if (slot < 0 || slot >= s->n_slots) return RD_E_STATE;
+        }
         CU(cudaMemcpy((char*)dst + (size_t)i * row_bytes, base + (size_t)slot * row_bytes, row_bytes, cudaMemcpyDeviceToHost));
     }
     return RD_OK;

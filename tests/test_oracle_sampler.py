@@ -316,3 +316,58 @@ def test_cached_sampler_equals_no_cache_recomputation(eps):
         assert np.abs(ia["logits"] - ib["logits"]).max() < 1e-9
         assert np.array_equal(ia["drafts"], ib["drafts"]) and ia["n_commit"] == ib["n_commit"]
     assert b.done and np.array_equal(a.committed(), b.committed())
+
+
+def test_one_latent_slot_turns_the_sampler_into_the_sequential_decoder():
+    """A pool with a single slot for hidden states (Appendix, "Larger Batch Sizes") leaves one position
+    in flight at a time; with the fixed exit it gets `window` steps of r' iterations on its own and is
+    then committed, which is the sequential decoder with r = window * r' (Section 3.3's identity),
+    token for token, in window steps per token."""
+    from helpers import SlotPoolModel
+    model, _ = make_oracle(SMALL, seed=4)
+    prompt = rd_inputs.make_prompt(7, SMALL["vocab"], seed=9)
+    sm = orc.Sampler(model, seed=5)
+    pool = SlotPoolModel(1)
+    sq = pool.start(sm, 0, prompt, 3, 6)
+    steps = 0
+    while not sq.done:
+        pool.drive(sm, [sq], 4, 2, 0.0)
+        assert len(sq.window) <= 1
+        steps += 1
+    model2, _ = make_oracle(SMALL, seed=4)
+    sm2 = orc.Sampler(model2, seed=5)
+    sq2 = sm2.prefill(0, prompt, 3, 6)
+    sm2.generate_ar(sq2, 8)
+    assert np.array_equal(sq.committed(), sq2.committed()) and steps == 6 * 4
+
+
+def test_a_large_enough_pool_changes_nothing_and_a_small_one_only_delays():
+    """With as many slots as batch x window the pooled schedule is the plain sampler; with fewer, every
+    sequence still finishes with its full budget and never holds more rows than the window."""
+    from helpers import SlotPoolModel
+    prompts = [rd_inputs.make_prompt(5 + 2 * b, SMALL["vocab"], seed=b) for b in range(3)]
+
+    def run(n_slots):
+        model, _ = make_oracle(SMALL, seed=2)
+        sm = orc.Sampler(model, seed=1)
+        pool = SlotPoolModel(n_slots)
+        seqs = [pool.start(sm, b, prompts[b], 2, 8) for b in range(3)]
+        steps = 0
+        while not all(sq.done for sq in seqs):
+            pool.drive(sm, seqs, 4, 1, 0.0)
+            assert sum(len(sq.window) for sq in seqs) <= n_slots and all(len(sq.window) <= 4 for sq in seqs)
+            steps += 1
+            assert steps < 500
+        return [sq.committed() for sq in seqs], steps
+
+    model, _ = make_oracle(SMALL, seed=2)
+    sm = orc.Sampler(model, seed=1)
+    plain = []
+    for b in range(3):
+        sq = sm.prefill(b, prompts[b], 2, 8)
+        sm.generate_df(sq, 4, 1, 0.0)
+        plain.append(sq.committed())
+    full, steps_full = run(12)
+    assert all(np.array_equal(a, b) for a, b in zip(full, plain)) and steps_full == 8 + 4 - 1
+    small, steps_small = run(5)
+    assert all(len(t) == len(p) for t, p in zip(small, plain)) and steps_small > steps_full
