@@ -196,23 +196,24 @@ __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restr
 }
 
 // x[row] = src[row] (+ resid[row]);  out[row] = g * x / sqrt(mean(x^2) + eps).
-// One cluster of NORM_CLUSTER blocks per row, grid (NORM_CLUSTER, rows): each block takes a run of
+// One cluster of CL blocks per row, grid (CL, rows): each block takes a run of
 // features, keeps its part of x in shared memory, and the blocks exchange their sums of squares
 // through distributed shared memory (added in block order).  `src` is a finished array or the
 // partial sums of the GEMM before (added here, in k order); with x_store, x is written out as the
 // new residual stream (x_store may alias resid).
-constexpr int NORM_CLUSTER = 8;
-template <typename TO>
+// CL blocks per row: 8 while few rows are in flight (latency), 2 for 128 rows and more (one wave of
+// blocks, each thread several groups of four).
+template <typename TO, int CL>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,
                size_t ldx, const float* __restrict__ g, int hidden, float eps, TO* __restrict__ out, size_t ldo,
                const int* __restrict__ row_pos) {
     extern __shared__ __align__(16) float xpart[];
     __shared__ float sm[32];
-    __shared__ float ss_all[NORM_CLUSTER];                       // every block's sum, pushed by its owner
+    __shared__ float ss_all[CL];                       // every block's sum, pushed by its owner
     // the gains are weights: they are fetched before the wait for the predecessor
     pdl_trigger();
-    const int chunk = ((hidden / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
+    const int chunk = ((hidden / 4 + CL - 1) / CL) * 4;
     const int m0 = blockIdx.x * chunk, m1 = min(hidden, m0 + chunk);
     constexpr int GMAX = 4;                                      // gains kept in registers per thread
     float gr[GMAX];
@@ -252,10 +253,10 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     // each block writes its sum into every block's table; after the cluster barrier all tables are
     // complete and nobody touches another block's memory again
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    if (threadIdx.x < NORM_CLUSTER) *cluster.map_shared_rank(&ss_all[blockIdx.x], threadIdx.x) = ss;
+    if (threadIdx.x < CL) *cluster.map_shared_rank(&ss_all[blockIdx.x], threadIdx.x) = ss;
     cluster.sync();
     float tot = 0.f;
-    for (int k = 0; k < NORM_CLUSTER; k++) tot += ss_all[k];
+    for (int k = 0; k < CL; k++) tot += ss_all[k];
     const float inv = 1.0f / sqrtf(tot / (float)hidden + eps);
 #pragma unroll
     for (int i = 0; i < GMAX; i++) {

@@ -340,7 +340,8 @@ template <typename F> static void want_max_carveout(F* kern) {
 }
 template <typename T> static void want_max_carveout_typed() {
     want_max_carveout(embed_kernel<T>);
-    want_max_carveout(rmsnorm_kernel<T>);
+    want_max_carveout(rmsnorm_kernel<T, 8>);
+    want_max_carveout(rmsnorm_kernel<T, 2>);
     want_max_carveout(concat_kernel<T>);
     want_max_carveout(gemm_simt_kernel<T, 1>);
     want_max_carveout(gemm_simt_kernel<T, 4>);
@@ -694,8 +695,14 @@ template <typename T> struct Eng {
     template <typename TO>
     static int norm(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
         const int h = s->m->cfg.hidden;
-        const size_t part = (size_t)((h / 4 + NORM_CLUSTER - 1) / NORM_CLUSTER) * 4;
-        LAUNCH_CLUSTER(s, rmsnorm_kernel<TO>, (NORM_CLUSTER, n_rows), 256, part * sizeof(float), NORM_CLUSTER, in.src, in.resid,
+        if (n_rows >= 128) return norm_cl<TO, 2>(s, in, x_store, g, out, n_rows);
+        return norm_cl<TO, 8>(s, in, x_store, g, out, n_rows);
+    }
+    template <typename TO, int CL>
+    static int norm_cl(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
+        const int h = s->m->cfg.hidden;
+        const size_t part = (size_t)((h / 4 + CL - 1) / CL) * 4;
+        LAUNCH_CLUSTER(s, (rmsnorm_kernel<TO, CL>), (CL, n_rows), 256, part * sizeof(float), CL, in.src, in.resid,
                        (size_t)h, x_store, (size_t)h, g, h, s->m->cfg.norm_eps, out, (size_t)h, s->row_pos);
         return RD_OK;
     }
@@ -765,7 +772,7 @@ template <typename T> struct Eng {
         const float* x_in = lazy ? s->x : in.src.plain;
         RowSource acc;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
-        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, n_rows >= 128 ? 4 : 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
                (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
