@@ -177,6 +177,17 @@ int rd_sync(rd_session* s);
  * sequence has produced max_new_tokens.  Either out pointer may be NULL. */
 int rd_committed(rd_session* s, int32_t seq, int32_t* n_tokens, int32_t* done);
 
+/* rd_poll_begin / rd_poll_end -- the same read without stalling the stream of steps.  rd_poll_begin
+ * enqueues, behind the steps enqueued so far, a device-to-host copy of the session's polled state
+ * (status word, |y_frozen| and done flag of every sequence) into one of two pinned buffers and returns
+ * its ticket (0 or 1) at once.  rd_poll_end waits for that copy only and reports sequence `seq`
+ * (seq = -1: *n_tokens = sum over the prefilled sequences, *done = all of them done).  A caller that
+ * enqueues step t+1 between the two calls for step t keeps the device busy while it reads; steps on
+ * finished sequences are no-ops, so running one step ahead is harmless.  At most two tickets are out
+ * at a time (STATE otherwise).  rd_poll_end returns TIMEOUT when the status word was set. */
+int rd_poll_begin(rd_session* s, int32_t* ticket);
+int rd_poll_end(rd_session* s, int32_t ticket, int32_t seq, int32_t* n_tokens, int32_t* done);
+
 /* rd_get_tokens -- copy up to `cap` tokens of y_frozen (prompt included) to host memory `dst`. */
 int rd_get_tokens(rd_session* s, int32_t seq, int32_t* dst, int32_t cap, int32_t* n_written);
 

@@ -18,7 +18,7 @@ EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
            "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining",
-           "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path"]
+           "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path", "rd_poll_begin", "rd_poll_end"]
 
 
 class RdConfig(C.Structure):
@@ -86,6 +86,8 @@ def lib():
         L.rd_debug_expire_next_wait.argtypes = [vp]
         L.rd_set_fused_swiglu.argtypes = [vp, i32]
         L.rd_set_attention_path.argtypes = [vp, i32]
+        L.rd_poll_begin.argtypes = [vp, C.POINTER(i32)]
+        L.rd_poll_end.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
         L.rd_profile_enable.argtypes = [vp, i32]
         L.rd_profile_read.argtypes = [vp, C.POINTER(RdProfile)]
         L.rd_strerror.argtypes = [C.c_int]
@@ -181,6 +183,16 @@ class Session:
     def committed(self, seq=0):
         n, d = C.c_int32(), C.c_int32()
         _check(lib().rd_committed(self.handle, seq, C.byref(n), C.byref(d)), "rd_committed")
+        return n.value, bool(d.value)
+
+    def poll_begin(self):
+        t = C.c_int32()
+        _check(lib().rd_poll_begin(self.handle, C.byref(t)), "rd_poll_begin")
+        return t.value
+
+    def poll_end(self, ticket, seq=-1):
+        n, d = C.c_int32(), C.c_int32()
+        _check(lib().rd_poll_end(self.handle, ticket, seq, C.byref(n), C.byref(d)), "rd_poll_end")
         return n.value, bool(d.value)
 
     def tokens(self, seq=0, out=None):

@@ -256,6 +256,10 @@ struct rd_session {
     size_t poll_ints = 0;    // status[4], n_committed[B], done[B] are one device block ...
     int* mirror = nullptr;   // ... mirrored in pinned host memory by one copy
     uint64_t enqueue_epoch = 1, mirror_epoch = 0;   // mirror is current while the two are equal
+    int* poll_mirror[2] = {nullptr, nullptr};       // pinned copies for rd_poll_begin / rd_poll_end
+    cudaEvent_t poll_ev[2] = {nullptr, nullptr};
+    bool poll_open[2] = {false, false};
+    int poll_next = 0;
     float *x = nullptr, *e = nullptr, *z = nullptr, *z_prev = nullptr;
     float *logits = nullptr, *delta = nullptr, *cos_t = nullptr, *sin_t = nullptr;
     float* tc_scratch = nullptr;   // partial sums of tiles whose K range is shared between CTAs
@@ -302,6 +306,10 @@ struct rd_session {
     uint64_t ctx_total = 0;   // host-side upper bound of sum over sequences of context length
     ~rd_session() {
         if (mirror) cudaFreeHost(mirror);
+        for (int i = 0; i < 2; i++) {
+            if (poll_mirror[i]) cudaFreeHost(poll_mirror[i]);
+            if (poll_ev[i]) cudaEventDestroy(poll_ev[i]);
+        }
         for (int i = 0; i < PROMPT_STAGES; i++) {
             if (prompt_stage[i]) cudaFreeHost(prompt_stage[i]);
             if (prompt_ev[i]) cudaEventDestroy(prompt_ev[i]);
@@ -488,6 +496,14 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
                 if (eh == cudaSuccess) eh = cudaEventCreateWithFlags(&s->prompt_ev[i], cudaEventDisableTiming);
             }
             if (eh != cudaSuccess) { rc = cuda_fail(eh, "prompt staging", __LINE__); break; }
+        }
+        {
+            cudaError_t eh = cudaSuccess;
+            for (int i = 0; i < 2 && eh == cudaSuccess; i++) {
+                eh = cudaHostAlloc((void**)&s->poll_mirror[i], s->poll_ints * sizeof(int), cudaHostAllocDefault);
+                if (eh == cudaSuccess) eh = cudaEventCreateWithFlags(&s->poll_ev[i], cudaEventDisableTiming);
+            }
+            if (eh != cudaSuccess) { rc = cuda_fail(eh, "poll mirrors", __LINE__); break; }
         }
         if ((rc = s->mem.get(&s->pf_e, (size_t)sc.max_context * h * sizeof(float)))) break;
         if ((rc = s->mem.get(&s->pf_s, (size_t)sc.max_context * h * sizeof(float)))) break;
@@ -1047,6 +1063,41 @@ extern "C" int rd_sync(rd_session* s) {
         s->mirror_epoch = s->enqueue_epoch;
     }
     return s->mirror[0] ? RD_E_TIMEOUT : RD_OK;
+}
+
+// Pipelined polling: begin enqueues a copy of the polled block (status word, |y_frozen| and done flag of
+// every sequence) behind the steps enqueued so far and returns at once; end waits for that copy only,
+// so the host can enqueue the next step before it reads the result of this one.
+extern "C" int rd_poll_begin(rd_session* s, int32_t* ticket) {
+    if (!s || !ticket) return RD_E_INVALID_ARG;
+    const int k = s->poll_next;
+    if (s->poll_open[k]) return RD_E_STATE;                 // both tickets are out: end one first
+    CU(cudaMemcpyAsync(s->poll_mirror[k], s->status, s->poll_ints * sizeof(int), cudaMemcpyDeviceToHost, s->stream));
+    CU(cudaEventRecord(s->poll_ev[k], s->stream));
+    s->poll_open[k] = true;
+    s->poll_next = k ^ 1;
+    *ticket = k;
+    return RD_OK;
+}
+extern "C" int rd_poll_end(rd_session* s, int32_t ticket, int32_t seq, int32_t* n_tokens, int32_t* done) {
+    if (!s || ticket < 0 || ticket > 1 || seq < -1 || seq >= s->sc.batch) return RD_E_INVALID_ARG;
+    if (!s->poll_open[ticket]) return RD_E_STATE;
+    CU(cudaEventSynchronize(s->poll_ev[ticket]));
+    const int* m = s->poll_mirror[ticket];
+    if (seq < 0) {
+        // all sequences: *n_tokens = sum of |y_frozen|, *done = 1 when every prefilled sequence is done
+        long long tot = 0;
+        int all = 1;
+        for (int b = 0; b < s->sc.batch; b++)
+            if (s->prefilled[b]) { tot += m[4 + b]; all &= m[4 + s->sc.batch + b] != 0; }
+        if (n_tokens) *n_tokens = (int32_t)tot;
+        if (done) *done = all;
+    } else {
+        if (n_tokens) *n_tokens = m[4 + seq];
+        if (done) *done = s->prefilled[seq] ? m[4 + s->sc.batch + seq] : 0;
+    }
+    s->poll_open[ticket] = false;
+    return m[0] ? RD_E_TIMEOUT : RD_OK;
 }
 
 extern "C" int rd_committed(rd_session* s, int32_t seq, int32_t* n_tokens, int32_t* done) {

@@ -136,3 +136,29 @@ def test_session_needs_the_models_device_current_and_read_ranges_do_not_wrap():
         assert fn(sess.handle, 1, 0, 0, 0, 62, 2, out.ctypes.data) == rd.RD_OK
     sess.close()
     gm.close()
+
+
+def test_pipelined_poll_reports_each_step_one_step_late():
+    """rd_poll_begin / rd_poll_end: the copy of the commit counters rides behind its step while the next
+    step is already enqueued; what it reports is that step's state, and a third open ticket is refused."""
+    shape, gm = _twin(seed=11)
+    W, N, L = 4, 6, 14
+    sess = rd.Session(gm, batch=1, max_context=64, max_window=W, max_new_tokens=N, seed=3)
+    sess.prefill(0, rd_inputs.make_prompt(L, shape["vocab"], seed=8), 2)
+    seen, pending = [], None
+    for t in range(1, N + W + 2):
+        sess.df_step(W, 1, 0.0)
+        ticket = sess.poll_begin()
+        if pending is not None:
+            seen.append(sess.poll_end(pending, 0))
+        pending = ticket
+    with pytest.raises(rd.RdError) as err:
+        a = sess.poll_begin()
+        sess.poll_begin()                                # both tickets out
+    assert err.value.code == rd.RD_E_STATE
+    sess.poll_end(a)
+    seen.append(sess.poll_end(pending, -1))
+    want = [(L + max(0, min(t, N + W - 1) - (W - 1)), t >= N + W - 1) for t in range(1, N + W + 2)]
+    assert seen == want
+    sess.close()
+    gm.close()
