@@ -327,7 +327,7 @@ attn_window_kernel(const GroupOrder order, const __nv_bfloat16* __restrict__ q_t
 // padding is needed and no bank conflicts arise.  The cache of one block is one 2-D tensor
 // [layers * sequences * heads * max_context rows, D]; a tile that reaches past a head's last position
 // reads rows of the next head (or zeros beyond the tensor), which the causal mask removes.
-// Thread 0 keeps STAGES - 1 tiles in flight beside the one being used: at the start of iteration i it
+// One thread keeps STAGES - 1 tiles in flight beside the one being used: at the start of iteration i it
 // refills the stage of tile i - 1 (released by every warp through an `empty` barrier) with tile
 // i - 1 + STAGES.  Every wait is
 // bounded; a wait that runs out raises the status word and the block goes on to the merge with
@@ -456,7 +456,7 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     const int seq = grp_index ? grp : row_seq[r0];          // pooled slots: group = sequence
     const int head_row0 = row_base + (seq * n_heads + hd) * max_context;   // row of this head's position 0
 
-    auto issue = [&](int it) {                              // thread 0: tile t0 + it into stage it % S
+    auto issue = [&](int it) {                              // issuing thread: tile t0 + it into stage it % S
         const int s = it % S;
         uint8_t* kdst = ring + s * C::STAGE_BYTES;
         uint8_t* vdst = kdst + T::BYTES;
@@ -472,8 +472,11 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
             att_tma_load_2d(vdst + T::NA * T::A_BYTES, &maps.v32, T::NA * 64, y, &full[s]);
         }
     };
+    // the thread that issues the copies: lane 0 of the LAST warp, which has no queries of its own when
+    // the group is small (one row per sequence in the sequential decoder) and then acts as a producer
+    const bool issuer = tid == NT - 32;
     int issued = 0;
-    if (tid == 0) {
+    if (issuer) {
         issued = min(S - 1, nt);
         for (int it = 0; it < issued; it++) issue(it);
     }
@@ -503,7 +506,7 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     bool ok = true;
     for (int it = 0; it < nt; it++) {
         const int s = it % S;
-        if (tid == 0 && issued < nt && ok) {
+        if (issuer && issued < nt && ok) {
             // keep S - 1 tiles in flight: the stage of tile it - 1 (or a fresh one) takes tile `issued`
             const int is = issued % S;
             if (issued >= S && !att_mbar_wait(&empty[is], ((issued / S) - 1) & 1)) { abort_s = 1; ok = false; }
@@ -579,7 +582,7 @@ attn_tma_kernel(const __grid_constant__ AttMaps maps, const GroupOrder order, co
     __syncthreads();
     if (abort_s) {
         // a wait ran out: let every copy this block issued land before its memory is reused or released
-        if (tid == 0) {
+        if (issuer) {
             for (int it = max(0, issued - S); it < issued; it++) att_mbar_wait(&full[it % S], (it / S) & 1);
             atomicExch(status, 1);
         }
