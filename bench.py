@@ -265,6 +265,8 @@ def run_ours(args):
         wl["temperature"] = args.temperature
     if args.top_p > 0.0:
         wl["top_p"] = args.top_p
+    if args.eps >= 0.0:
+        wl["eps"] = args.eps
     if args.window > 0:
         wl["window"] = args.window
     if args.inner > 0:
@@ -658,6 +660,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--ar-tokens", type=int, default=24)
     ap.add_argument("--window", type=int, default=0, help="override the workload's window (sweeps)")
+    ap.add_argument("--eps", type=float, default=-1.0, help="override the workload's exit threshold (0: fixed exit)")
     ap.add_argument("--inner", type=int, default=0, help="override the workload's inner iterations per step (sweeps)")
     ap.add_argument("--prefill-r", type=int, default=0, help="override the workload's prefill recurrence (profiling aid)")
     ap.add_argument("--temperature", type=float, default=-1.0, help="override the workload's sampling temperature (sweeps)")

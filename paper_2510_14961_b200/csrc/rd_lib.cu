@@ -712,7 +712,7 @@ template <typename T> struct Eng {
     template <typename TO>
     static int norm(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
         const int h = s->m->cfg.hidden;
-        if (n_rows >= 128) return norm_cl<TO, 2>(s, in, x_store, g, out, n_rows);
+        if (n_rows >= 128) return norm_cl<TO, 2>(s, in, x_store, g, out, n_rows);   // (4-block clusters at 256 rows: no difference in an A/B)
         return norm_cl<TO, 8>(s, in, x_store, g, out, n_rows);
     }
     template <typename TO, int CL>
@@ -792,7 +792,7 @@ template <typename T> struct Eng {
         const float* x_in = lazy ? s->x : in.src.plain;
         RowSource acc;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
-        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, n_rows >= 128 ? 4 : 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
                (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;

@@ -37,6 +37,28 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     const size_t in_slot = ((size_t)(ft & ((1u << d.mt_shift) - 1)) * d.bn + (size_t)(r % d.bn)) * 128 + (m & 127);
     const float* base = d.scratch + in_slot;
     const size_t slot_elems = ((size_t)d.bn * 128) << d.mt_shift;
+    if (d.bn >= 128) {
+        // Many rows in flight (batched steps, prefill): the readers are bound by their instruction count
+        // there, so the slot addresses come from one division.  CTA g_lo may have started in an earlier
+        // tile; every later CTA of the tile starts inside it, so its first slot is the tile's.  Same slots,
+        // same order of addition as below: the same bits.
+        const unsigned first0 = ((unsigned)g_lo * (unsigned)d.per) / (unsigned)d.kb;
+        const size_t cta_stride = (size_t)d.max_seg * slot_elems;
+        float4 acc = __ldcg(reinterpret_cast<const float4*>(base + (size_t)g_lo * cta_stride + (size_t)(tile - first0) * slot_elems));
+        const float* q = base + (size_t)(g_lo + 1) * cta_stride;
+        for (int g = g_lo + 1; g <= g_hi; g += 4, q += 4 * cta_stride) {
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (g + j <= g_hi) v[j] = __ldcg(reinterpret_cast<const float4*>(q + (size_t)j * cta_stride));
+            }
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+                if (g + j <= g_hi) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+        }
+        return acc;
+    }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     // up to eight slots are requested together (one round trip to L2), then added in ascending k order
     for (int gb = g_lo; gb <= g_hi; gb += 8) {
