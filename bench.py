@@ -414,6 +414,7 @@ def run_ours(args):
     whole_generation_tok_s = gen_tok / (gen_ms / 1e3)
 
     # ---- per-kernel roofline: event pairs around every GEMM / attention launch -----------------
+    rows_full = B * W
     prefill(sess)
     for _ in range(W + 2):                  # reach the full window
         sess.df_step(W, wl["inner"], wl["eps"])
@@ -425,6 +426,22 @@ def run_ours(args):
     prof = sess.profile_read()
     sess.profile_enable(False)
     gemm_gbs = prof["gemm_weight_bytes"] / (prof["gemm_ms"] * 1e-3) / 1e9 if prof["gemm_ms"] > 0 else 0.0
+    # the same GEMM launches as a chain of their own (the launch mode of the timed steps: programmatic
+    # dependent launches, no event between them), timed with one event pair around 20 steps' worth
+    chain = None
+    try:
+        sess.gemm_sequence(rows_full, 2)                    # warm
+        sess.sync()
+        with torch.cuda.stream(stream):
+            ev0.record(stream)
+            chain_bytes, chain_launches = sess.gemm_sequence(rows_full, 20)
+            ev1.record(stream)
+        sess.sync()
+        chain_ms = ev0.elapsed_time(ev1)
+        chain = {"achieved": chain_bytes / (chain_ms * 1e-3) / 1e9, "launches": chain_launches,
+                 "avg_us": 1e3 * chain_ms / chain_launches, "bytes_per_launch": chain_bytes / chain_launches}
+    except rd.RdError:
+        pass                                                # float32 configuration: no tensor-core GEMM path
     attn_gbs = prof["attn_kv_bytes"] / (prof["attn_ms"] * 1e-3) / 1e9 if prof["attn_ms"] > 0 else 0.0
     tc_launches = sess.stats()["tc_gemm_launches"]
     # step roofline for the steps that were timed: algorithmic bytes and FLOPs as the library's
@@ -498,6 +515,21 @@ def run_ours(args):
     e2e_tok_s = got_all / e2e_s_max
     e2e.close()
 
+    # Dominant kernel: the weight-streaming GEMM.  `achieved` is measured in the launch mode of the timed
+    # steps (a chain of programmatic dependent launches: the 34 GEMM launches of a step back to back, 20
+    # steps' worth inside one event pair); `alone` is the same launches each inside its own event pair
+    # during real steps (the pair breaks the chain, so the launch gap and a cold start are included).
+    alone = {"achieved": gemm_gbs, "frac": gemm_gbs / peaks["hbm_gbs"], "launches": prof["gemm_launches"],
+             "avg_us": 1e3 * prof["gemm_ms"] / max(prof["gemm_launches"], 1),
+             "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1)}
+    best = chain if chain else alone
+    roofline = {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections of the step)",
+                "achieved": best["achieved"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": best["achieved"] / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(args.workload),
+                "launches": best["launches"], "avg_us": best["avg_us"], "bytes_per_launch": best["bytes_per_launch"],
+                "how": "GEMM launches of 20 steps as one chain of programmatic dependent launches, one CUDA-event pair"
+                       if chain else "one CUDA-event pair around every GEMM launch of 20 steps",
+                "alone": alone, "peak_source": peaks["source"]}
     line = {
         "metric": "generated tok/s at 1 B200, DF sampler vs AR recurrence; % of step roofline",
         "value": df_tok_s, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": warm,
@@ -528,12 +560,7 @@ def run_ours(args):
                           "df_frac": t_roof * 1e3 / ms_per_step,
                           "ar_t_roof_ms": ar_roof * 1e3, "ar_frac": ar_roof / (ar_ms / n_ar / 1e3),
                           "peak_source": peaks["source"]},
-        "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections of the step)",
-                     "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(args.workload),
-                     "launches": prof["gemm_launches"], "avg_us": 1e3 * prof["gemm_ms"] / max(prof["gemm_launches"], 1),
-                     "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
-                     "peak_source": peaks["source"]},
+        "roofline": roofline,
         "attention": {"achieved_gbs": attn_gbs, "launches": prof["attn_launches"],
                       "avg_us": 1e3 * prof["attn_ms"] / max(prof["attn_launches"], 1)},
         "kernel_time_shares": {k: prof[k + "_ms"] / max(prof["gemm_ms"] + prof["attn_ms"] + prof["other_ms"], 1e-9)

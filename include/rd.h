@@ -267,6 +267,16 @@ typedef struct {
 int rd_profile_enable(rd_session* s, int32_t on);
 int rd_profile_read(rd_session* s, rd_profile_t* out);
 
+/* rd_debug_gemm_sequence -- measurement aid: enqueues, `reps` times, the GEMM launches of one decode
+ * step with one inner iteration (every layer's QKV, out, gate/up and down projection, the adapter, the
+ * head; same shapes, operands, row tile and launch mode as in a step) with nothing between them, on
+ * `n_rows` rows of the session's activation buffers as they stand (results unused; the session's
+ * sequences are not touched, but a step enqueued later recomputes its activations anyway).  Timed
+ * with events on the session's stream it gives the GEMM's launch duration inside a chain of launches,
+ * without the gap that an event pair around a single launch adds.  *weight_bytes = algorithmic weight
+ * bytes of the enqueued launches, *launches = their number.  RD_BF16 tensor-core path only (STATE). */
+int rd_debug_gemm_sequence(rd_session* s, int32_t n_rows, int32_t reps, uint64_t* weight_bytes, int32_t* launches);
+
 /* rd_set_gemm_path -- 0: SIMT kernels everywhere; 1 (default for RD_BF16): tcgen05 tensor-core
  * GEMMs where the shape allows, tiles of 128 and 256 rows on CTA pairs (one MMA of 256 features over
  * two SMs); 2: as 1 with those tiles on single CTAs.  For measurement and parity tests. */

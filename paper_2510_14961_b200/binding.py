@@ -18,7 +18,8 @@ EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_
            "rd_df_step", "rd_sync", "rd_committed", "rd_get_tokens", "rd_last_step_rows", "rd_debug_read",
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
            "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining",
-           "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path", "rd_poll_begin", "rd_poll_end"]
+           "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path", "rd_poll_begin", "rd_poll_end",
+           "rd_debug_gemm_sequence"]
 
 
 class RdConfig(C.Structure):
@@ -86,6 +87,7 @@ def lib():
         L.rd_debug_expire_next_wait.argtypes = [vp]
         L.rd_set_fused_swiglu.argtypes = [vp, i32]
         L.rd_set_attention_path.argtypes = [vp, i32]
+        L.rd_debug_gemm_sequence.argtypes = [vp, i32, i32, C.POINTER(C.c_uint64), C.POINTER(i32)]
         L.rd_poll_begin.argtypes = [vp, C.POINTER(i32)]
         L.rd_poll_end.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
         L.rd_profile_enable.argtypes = [vp, i32]
@@ -255,6 +257,12 @@ class Session:
 
     def set_fused_swiglu(self, on):
         _check(lib().rd_set_fused_swiglu(self.handle, 1 if on else 0), "rd_set_fused_swiglu")
+
+    def gemm_sequence(self, n_rows, reps=1):
+        """Measurement aid: the GEMM launches of a decode step, back to back; returns (weight bytes, launches)."""
+        b, n = C.c_uint64(), C.c_int32()
+        _check(lib().rd_debug_gemm_sequence(self.handle, n_rows, reps, C.byref(b), C.byref(n)), "rd_debug_gemm_sequence")
+        return b.value, n.value
 
     def expire_next_wait(self):
         """Test aid: the next tensor-core GEMM launch lets one bounded wait run out (RD_E_TIMEOUT at the next sync)."""

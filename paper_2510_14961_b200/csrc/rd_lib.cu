@@ -952,6 +952,26 @@ template <typename T> struct Eng {
         return RD_OK;
     }
 
+    // The GEMM launches of one decode step (inner_iters = 1), in the step's order and launch mode, with
+    // nothing between them: prelude layers, adapter, core layers, coda layers, head.  Operands are the
+    // session's activation buffers as they stand; the results are not used.  Measurement aid.
+    static int gemm_sequence(rd_session* s, int n_rows) {
+        const rd_config& c = s->m->cfg;
+        const int h = c.hidden, I = c.mlp_inner;
+        RowSource acc;
+        bool fused = false;
+        for (int blk = 0; blk < 3; blk++) {
+            if (blk == 1) RD_TRY(gemm(s, (T*)s->act_2h, 2 * h, &s->t_act_2h, (T*)s->m->adapter, &s->m->t_adapter, 2 * h, h, n_rows, &acc));
+            for (const LayerW& L : s->m->layers[blk]) {
+                RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
+                RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wo, &L.t_o, h, h, n_rows, &acc));
+                RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wgu, &L.t_gu, h, 2 * I, n_rows, &acc, (T*)s->act_i, &fused));
+                RD_TRY(gemm(s, (T*)s->act_i, I, &s->t_act_i, (T*)L.wd, &L.t_d, I, h, n_rows, &acc));
+            }
+        }
+        return gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, n_rows, &acc);
+    }
+
     static int prefill_passes(rd_session* s, int seq, int n, int r, float* e_all, float* s_all) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
@@ -1289,6 +1309,19 @@ extern "C" int rd_debug_expire_next_wait(rd_session* s) {
     if (!s) return RD_E_INVALID_ARG;
     if (!(s->gemm_path >= 1 && s->m->tc_ok && s->tc_scratch)) return RD_E_STATE;
     s->expire_next_wait = true;
+    return RD_OK;
+}
+
+extern "C" int rd_debug_gemm_sequence(rd_session* s, int32_t n_rows, int32_t reps, uint64_t* weight_bytes, int32_t* launches) {
+    if (!s || n_rows < 1 || n_rows > s->R || reps < 1) return RD_E_INVALID_ARG;
+    if (s->m->cfg.dtype != RD_BF16 || s->gemm_path < 1 || !s->m->tc_ok) return RD_E_STATE;
+    const rd_config& c = s->m->cfg;
+    const uint64_t h = c.hidden, per_layer = 4 * h * h + 3 * h * (uint64_t)c.mlp_inner;
+    const int n_layers = c.n_prelude + c.n_core + c.n_coda;
+    for (int i = 0; i < reps; i++) RD_TRY(Eng<bf16>::gemm_sequence(s, n_rows));
+    s->enqueue_epoch++;
+    if (weight_bytes) *weight_bytes = (uint64_t)reps * (n_layers * per_layer + 2 * h * h + (uint64_t)c.vocab * h) * s->m->esz;
+    if (launches) *launches = reps * (4 * n_layers + 2);
     return RD_OK;
 }
 
