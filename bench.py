@@ -298,7 +298,7 @@ def run_ours(args):
         if args.unfused_swiglu:
             ses.set_fused_swiglu(False)     # A/B: gate/up leaves partial sums, SwiGLU in a kernel of its own
         if args.attention_path >= 0:
-            ses.set_attention_path(args.attention_path)   # A/B: 2 TMA ring (default), 1 cp.async, 0 one block per row
+            ses.set_attention_path(args.attention_path)   # A/B: 3 default, 2 mma.sync prefill, 1 cp.async, 0 one block per row
         if args.unchained:
             ses.set_launch_chaining(False)  # A/B: ordinary stream-ordered launches
         return ses
@@ -548,7 +548,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (weights streamed per step: %.2f GB)" % (step_b / 1e9),
                    "multi_gpu": "replicas only (no data-path collective)",
                    "variant": {"fused_swiglu": not args.unfused_swiglu, "chained_launches": not args.unchained,
-                               "attention_path": 2 if args.attention_path < 0 else args.attention_path}},
+                               "attention_path": 3 if args.attention_path < 0 else args.attention_path}},
         "df_tok_s": df_tok_s, "ar_tok_s": ar_tok_s, "df_over_ar": df_tok_s / ar_tok_s if ar_tok_s else None,
         "ar_tokens_timed": n_ar, "ar_ms_per_token": ar_ms / n_ar,
         "prefill": {"seconds": prefill_s, "flops": pf_flops, "tflops": pf_flops / prefill_s / 1e12,
@@ -694,7 +694,7 @@ def main():
     ap.add_argument("--top-p", type=float, default=0.0, help="top-p of Sample (sweeps; needs a temperature > 0)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--unfused-swiglu", action="store_true", help="A/B: SwiGLU as a separate kernel")
-    ap.add_argument("--attention-path", type=int, default=-1, help="A/B: 2 TMA ring (default), 1 cp.async, 0 SIMT")
+    ap.add_argument("--attention-path", type=int, default=-1, help="A/B: 3 default (TMA ring; tcgen05 prefill), 2 without the tcgen05 prefill kernel, 1 cp.async, 0 SIMT")
     ap.add_argument("--unchained", action="store_true", help="A/B: no programmatic dependent launch")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

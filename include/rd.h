@@ -287,8 +287,10 @@ int rd_set_gemm_path(rd_session* s, int32_t path);
  * 0: ordinary stream-ordered launches.  Results are identical; for measurement and tests. */
 int rd_set_launch_chaining(rd_session* s, int32_t on);
 
-/* rd_set_attention_path -- 2 (default for RD_BF16 with head_dim 64, 96 or 128): windowed tensor-core
- * attention with K and V brought in by TMA through a ring of barrier-guarded stages (groups of at most
+/* rd_set_attention_path -- 3 (default for RD_BF16 with head_dim 64, 96 or 128): as 2, and prefill
+ * (groups of 128 consecutive prompt rows) with both products on tcgen05, S and O in tensor memory;
+ * 2: windowed tensor-core attention (mma.sync) with K and V brought in by TMA through a ring of
+ * barrier-guarded stages (groups of at most
  * 8 rows, e.g. the sequential decoder's one row per sequence, take the cp.async kernel); 1: the same
  * arithmetic with K and V brought in by cp.async, double buffered; 0: one block per (row, head).
  * For measurement (A/B) and tests.  STATE when the model cannot take the requested path. */

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librd_b200.so")
 SOURCES = ["rd_lib.cu"]
-HEADERS = ["rd_common.cuh", "rd_partial.cuh", "rd_kernels.cuh", "rd_gemm_tc.cuh", "rd_attn.cuh", os.path.join("..", "..", "include", "rd.h")]
+HEADERS = ["rd_common.cuh", "rd_partial.cuh", "rd_kernels.cuh", "rd_gemm_tc.cuh", "rd_attn.cuh", "rd_attn_tc.cuh", os.path.join("..", "..", "include", "rd.h")]
 
 
 def _stale() -> bool:

@@ -1,0 +1,285 @@
+// Causal prefill attention on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// Prefill (Section 3.3: all prompt positions iterate the recurrence together) attends 128 consecutive
+// prompt rows of one sequence to the cache entries 0..p of that sequence.  With 128 queries per K/V
+// tile the arithmetic (4 * 128 * head_dim FLOPs per key) is past what mma.sync sustains, so here both
+// products run as tcgen05.mma with the accumulators in tensor memory:
+//   S[128 q, 64 keys] = Q K^T        A = Q (K-major), B = K tile (K-major), M = 128, N = 64
+//   O[128 q, D]      += P V          A = P (bf16, written to shared memory by the softmax warps),
+//                                    B = V tile as it lies in the cache, [key][d] (MN-major), N = 64 (+ 32)
+// One CTA per (group of 128 rows, head), no key splits: a group's keys are walked tile by tile.
+//   warp 0 / lane 0   TMA producer: Q once, then K and V tiles through a ring of stages
+//   warp 1 / lane 0   issues the MMAs; tcgen05.commit signals the softmax warps and frees stages
+//   warps 2-5         one query row per thread (TMEM lane = row): S from TMEM, causal mask, online
+//                     softmax in float32 (log2 domain), P to shared memory in the 128-byte swizzle,
+//                     then the tile's P V from TMEM into the running output in registers
+// Q, K, V sub-tiles are the ones of rd_attn.cuh (64 columns with the 128-byte swizzle, 32 with the
+// 64-byte swizzle for the last third of a 96-wide head), written by TMA and described to the MMA by
+// shared-memory descriptors.  Every wait is bounded; on time-out the kernel raises the status word,
+// lets its copies land, frees its TMEM and returns.
+#pragma once
+#include "rd_attn.cuh"
+#include "rd_gemm_tc.cuh"
+
+namespace rd {
+
+constexpr int ATC_Q = 128;          // queries per CTA (UMMA M)
+constexpr int ATC_THREADS = 192;
+constexpr int ATC_STAGES = 2;        // 91 KB at head_dim 96: two CTAs per SM (one's MMAs run under the other's softmax)
+
+// K-major tile with rows of 64 bytes (32 bf16), 64-byte swizzle: 8-row groups 512 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k64(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
+}
+// MN-major operand ([k][n] in memory, n contiguous): rows of 128 bytes (64 n) with the 128-byte swizzle,
+// 8-row (8 k) groups 1024 bytes apart; rows of 64 bytes (32 n) with the 64-byte swizzle, groups 512 apart.
+__device__ __forceinline__ uint64_t umma_desc_mn128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t umma_desc_mn64(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
+}
+// instruction descriptor with B given MN-major (bit 16)
+__host__ __device__ constexpr uint32_t umma_idesc_bmn(int bn) { return umma_idesc(bn) | (1u << 16); }
+
+template <int D> struct AtcCfg {
+    using T = AttTile<D>;
+    static constexpr int NA = T::NA, NB = T::NB;
+    static constexpr int QA_BYTES = ATC_Q * 128, QB_BYTES = ATC_Q * 64;       // Q sub-tiles (128 rows)
+    static constexpr int Q_BYTES = NA * QA_BYTES + NB * QB_BYTES;
+    static constexpr int KV_STAGE = 2 * T::BYTES;                             // K tile, V tile of 64 keys
+    static constexpr int P_BYTES = ATC_Q * 128;                               // P: 128 rows x 64 keys bf16
+    static constexpr int SMEM = 1024 + Q_BYTES + ATC_STAGES * KV_STAGE + P_BYTES + 256;
+    static constexpr int TMEM_COLS = 256;                                     // S 64 | O 64 (+64) | O 32
+    static constexpr int O_COL = 64;
+};
+
+struct AtcMaps {
+    CUtensorMap q64, q32;             // boxes of 128 rows x 64 / 32 columns over the query buffer [rows, hidden]
+    AttMaps kv;                       // boxes of 64 keys over the K and the V cache of the block
+};
+
+template <int D>
+__global__ void __launch_bounds__(ATC_THREADS, 2)
+attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                       int n_rows, int row_base, int n_heads, int max_context, int hidden, float scale_log2,
+                       __nv_bfloat16* __restrict__ out, int* __restrict__ status) {
+    using C = AtcCfg<D>;
+    using T = AttTile<D>;
+    constexpr int S = ATC_STAGES;
+    extern __shared__ uint8_t atc_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)atc_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* Qs = smem;
+    uint8_t* ring = Qs + C::Q_BYTES;
+    uint8_t* Ps = ring + S * C::KV_STAGE;
+    uint64_t* q_full = (uint64_t*)(Ps + C::P_BYTES);
+    uint64_t* kv_full = q_full + 1;           // [S]
+    uint64_t* kv_empty = kv_full + S;         // [S]
+    uint64_t* s_full = kv_empty + S;
+    uint64_t* p_full = s_full + 1;
+    uint64_t* o_full = p_full + 1;
+    uint64_t* o_free = o_full + 1;
+    uint32_t* tmem_slot = (uint32_t*)(o_free + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    __shared__ int kv_len_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hd = blockIdx.x, r0 = blockIdx.y * ATC_Q;
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < S; s++) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        mbar_init(s_full, 1); mbar_init(p_full, ATC_Q); mbar_init(o_full, 1); mbar_init(o_free, ATC_Q);
+        *abort_flag = 0;
+        kv_len_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    pdl_enter();
+    // positions of the group's rows (consecutive rows of the row table); kv_len = 1 + the largest
+    int my_pos = -1;
+    if (warp >= 2) {
+        const int r = r0 + (warp & 3) * 32 + lane;
+        my_pos = r < n_rows ? row_pos[r] : -1;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp >= 2) {
+        const int wmax = __reduce_max_sync(0xffffffffu, my_pos);
+        if (lane == 0 && wmax >= 0) atomicMax(&kv_len_s, wmax + 1);
+    }
+    __syncthreads();
+    const int kv_len = kv_len_s;
+    const int nt = (kv_len + ATT_KT - 1) / ATT_KT;
+    const uint32_t tmem_base = *tmem_slot;
+    const int seq = row_seq[min(r0, n_rows - 1)];
+    const int head_row0 = row_base + (seq * n_heads + hd) * max_context;
+
+    if (warp == 0) {
+        if (lane == 0 && nt > 0) {
+            // ---- TMA producer ----
+            mbar_expect_tx(q_full, C::Q_BYTES);
+#pragma unroll
+            for (int a = 0; a < C::NA; a++) tma_load_2d(Qs + a * C::QA_BYTES, &maps.q64, hd * D + a * 64, r0, q_full);
+            if (C::NB) tma_load_2d(Qs + C::NA * C::QA_BYTES, &maps.q32, hd * D + C::NA * 64, r0, q_full);
+            int issued = 0;
+            for (int t = 0; t < nt; t++) {
+                const int s = t % S;
+                if (t >= S && (*abort_flag || !mbar_wait(&kv_empty[s], ((t / S) - 1) & 1))) { *abort_flag = 1; break; }
+                uint8_t* kdst = ring + s * C::KV_STAGE;
+                uint8_t* vdst = kdst + T::BYTES;
+                const int y = head_row0 + t * ATT_KT;
+                mbar_expect_tx(&kv_full[s], C::KV_STAGE);
+#pragma unroll
+                for (int a = 0; a < T::NA; a++) {
+                    tma_load_2d(kdst + a * T::A_BYTES, &maps.kv.k64, a * 64, y, &kv_full[s]);
+                    tma_load_2d(vdst + a * T::A_BYTES, &maps.kv.v64, a * 64, y, &kv_full[s]);
+                }
+                if (T::NB) {
+                    tma_load_2d(kdst + T::NA * T::A_BYTES, &maps.kv.k32, T::NA * 64, y, &kv_full[s]);
+                    tma_load_2d(vdst + T::NA * T::A_BYTES, &maps.kv.v32, T::NA * 64, y, &kv_full[s]);
+                }
+                issued = t + 1;
+            }
+            if (*abort_flag) {
+                mbar_wait(q_full, 0);
+                for (int t = max(0, issued - S); t < issued; t++) mbar_wait(&kv_full[t % S], (t / S) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && nt > 0) {
+            // ---- MMA issuer ----
+            constexpr uint32_t idesc_s = umma_idesc(ATT_KT);            // S: N = 64 keys
+            constexpr uint32_t idesc_o64 = umma_idesc_bmn(64);          // O columns of a 64-wide V sub-tile
+            constexpr uint32_t idesc_o32 = umma_idesc_bmn(32);
+            const uint32_t q0 = smem_u32(Qs), p0 = smem_u32(Ps);
+            bool ok = mbar_wait(q_full, 0);
+            auto issue_qk = [&](int t) {
+                const uint32_t k0 = smem_u32(ring + (t % S) * C::KV_STAGE);
+                tc_fence_after();
+                int step = 0;
+#pragma unroll
+                for (int a = 0; a < C::NA; a++)
+#pragma unroll
+                    for (int k = 0; k < 4; k++, step++)
+                        umma_bf16(tmem_base, umma_desc_k128(q0 + a * C::QA_BYTES) + (uint64_t)(k * 2),
+                                  umma_desc_k128(k0 + a * T::A_BYTES) + (uint64_t)(k * 2), idesc_s, step ? 1u : 0u);
+                if (C::NB) {
+#pragma unroll
+                    for (int k = 0; k < 2; k++, step++)
+                        umma_bf16(tmem_base, umma_desc_k64(q0 + C::NA * C::QA_BYTES) + (uint64_t)(k * 2),
+                                  umma_desc_k64(k0 + T::NA * T::A_BYTES) + (uint64_t)(k * 2), idesc_s, step ? 1u : 0u);
+                }
+                umma_commit(s_full);
+            };
+            if (ok) ok = mbar_wait(&kv_full[0], 0);
+            if (ok) issue_qk(0);
+            for (int t = 0; t < nt && ok; t++) {
+                const int s = t % S;
+                if (*abort_flag || !mbar_wait(p_full, t & 1)) { ok = false; break; }          // P(t) in shared memory, S free
+                if (t > 0 && !mbar_wait(o_free, (t - 1) & 1)) { ok = false; break; }          // O(t-1) read out of TMEM
+                tc_fence_after();
+                const uint32_t v0 = smem_u32(ring + s * C::KV_STAGE + T::BYTES);
+#pragma unroll
+                for (int a = 0; a < T::NA; a++)
+#pragma unroll
+                    for (int k = 0; k < 4; k++)          // 16 keys per MMA: 16 rows of the V sub-tile further on
+                        umma_bf16(tmem_base + (uint32_t)(C::O_COL + a * 64), umma_desc_k128(p0) + (uint64_t)(k * 2),
+                                  umma_desc_mn128(v0 + a * T::A_BYTES + k * 2048), idesc_o64, k ? 1u : 0u);
+                if (T::NB) {
+#pragma unroll
+                    for (int k = 0; k < 4; k++)
+                        umma_bf16(tmem_base + (uint32_t)(C::O_COL + T::NA * 64), umma_desc_k128(p0) + (uint64_t)(k * 2),
+                                  umma_desc_mn64(v0 + T::NA * T::A_BYTES + k * 1024), idesc_o32, k ? 1u : 0u);
+                }
+                umma_commit(&kv_empty[s]);               // K and V of this stage have been read
+                umma_commit(o_full);
+                if (t + 1 < nt) {
+                    if (*abort_flag || !mbar_wait(&kv_full[(t + 1) % S], ((t + 1) / S) & 1)) { ok = false; break; }
+                    issue_qk(t + 1);                     // runs while the softmax warps take O(t)
+                }
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else {
+        // ---- softmax warps: thread = query row ----
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;                 // row of the group = TMEM lane
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
+        float m = -INFINITY, l = 0.f;
+        float o[D];
+#pragma unroll
+        for (int j = 0; j < D; j++) o[j] = 0.f;
+        bool ok = true;
+        for (int t = 0; t < nt && ok; t++) {
+            if (*abort_flag || !mbar_wait(s_full, t & 1)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t sr[64];
+            tmem_ld32(t_lane, sr);
+            tmem_ld32(t_lane + 32, sr + 32);
+            const int key0 = t * ATT_KT;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 64; j++) {
+                const float v = (key0 + j <= my_pos) ? __uint_as_float(sr[j]) * scale_log2 : -INFINITY;
+                sr[j] = __float_as_uint(v);
+                mx = fmaxf(mx, v);
+            }
+            const float mn = fmaxf(m, mx);
+            const float u = mn == -INFINITY ? 0.f : mn;
+            const float corr = exp2f(m - u);
+            m = mn;
+            float sum = 0.f;
+            // P row: 64 bf16 = 8 chunks of 16 bytes, chunk c at (c ^ (row & 7)) of the row's 128 bytes
+            uint8_t* prow = Ps + row * 128;
+#pragma unroll
+            for (int c = 0; c < 8; c++) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    const float p0 = exp2f(__uint_as_float(sr[c * 8 + 2 * q]) - u), p1 = exp2f(__uint_as_float(sr[c * 8 + 2 * q + 1]) - u);
+                    sum += p0 + p1;
+                    w[q] = pack_bf16(p0, p1);
+                }
+                *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            l = l * corr + sum;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // P visible to the tensor core's reads
+            tc_fence_before();
+            mbar_arrive(p_full);
+            if (!mbar_wait(o_full, t & 1)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < D; c += 32) {
+                uint32_t orow[32];
+                tmem_ld32(t_lane + (uint32_t)(C::O_COL + c), orow);
+#pragma unroll
+                for (int j = 0; j < 32; j++) o[c + j] = o[c + j] * corr + __uint_as_float(orow[j]);
+            }
+            tc_fence_before();
+            mbar_arrive(o_free);
+        }
+        if (!ok) *abort_flag = 1;
+        if (ok && my_pos >= 0) {
+            const float inv = l > 0.f ? 1.0f / l : 0.f;
+            __nv_bfloat16* dst = out + (size_t)(r0 + row) * hidden + hd * D;
+#pragma unroll
+            for (int c = 0; c < D; c += 8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) w[q] = pack_bf16(o[c + 2 * q] * inv, o[c + 2 * q + 1] * inv);
+                *reinterpret_cast<uint4*>(dst + c) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) atomicExch(status, 1);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(*tmem_slot, C::TMEM_COLS);
+    }
+}
+
+}  // namespace rd

@@ -14,6 +14,7 @@
 
 #include "../../include/rd.h"
 #include "rd_attn.cuh"
+#include "rd_attn_tc.cuh"
 #include "rd_gemm_tc.cuh"
 #include "rd_kernels.cuh"
 
@@ -288,6 +289,8 @@ struct rd_session {
     int attn_path = 0;          // 1: windowed tensor-core attention (bf16, head_dim 64/96/128), K/V by cp.async;
                                 // 2: the same fed by TMA through an mbarrier ring (needs the tensor maps below)
     bool att_maps_ok = false, attn_capable = false;
+    CUtensorMap q_map64, q_map32;   // the query buffer [rows, hidden] in boxes of 128 rows x 64 / 32 columns
+    bool q_maps_ok = false;
     AttMaps att_maps[3];        // per block: boxes of 64 and 32 columns over the K and the V cache
     void *act_h = nullptr, *act_2h = nullptr, *act_i = nullptr, *q_t = nullptr;
     void *Kc[3] = {nullptr, nullptr, nullptr}, *Vc[3] = {nullptr, nullptr, nullptr};
@@ -370,6 +373,7 @@ template <int D> static cudaError_t attn_configure_d() {
     set(attn_tma_kernel<D, 32, 4>, AttTmaCfg<D, 4>::SMEM);
     set(attn_tma_kernel<D, 64, 4>, AttTmaCfg<D, 4>::SMEM);
     set(attn_tma_kernel<D, 64, 8>, AttTmaCfg<D, 8>::SMEM);
+    set(attn_prefill_tc_kernel<D>, AtcCfg<D>::SMEM);
     return e;
 }
 // Function attributes (shared-memory opt-in, carve-out preference) are kept per device: they are
@@ -410,6 +414,20 @@ static int attn_encode(CUtensorMap* map, const void* ptr, unsigned long long row
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
     const cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)ATT_KT};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RD_OK : RD_E_CUDA;
+}
+
+// The query buffer [rows, hidden] in boxes of 128 rows x `cols` columns (one head's sub-tile of a group).
+static int q_encode(CUtensorMap* map, const void* ptr, unsigned long long rows, int hidden, int cols) {
+    if (!g_encode_tiled) return RD_E_STATE;
+    if (((uintptr_t)ptr & 15) != 0 || (hidden * 2) % 16 != 0) return RD_E_INVALID_ARG;
+    const cuuint64_t dims[2] = {(cuuint64_t)hidden, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)hidden * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)ATC_Q};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
@@ -563,6 +581,11 @@ extern "C" int rd_session_create(const rd_model* m, const rd_session_config* scp
             }
             s->att_maps_ok = maps_ok;
             if (maps_ok) s->attn_path = 2;
+            if (maps_ok) {
+                s->q_maps_ok = q_encode(&s->q_map64, s->q_t, R, c.hidden, 64) == RD_OK &&
+                               q_encode(&s->q_map32, s->q_t, R, c.hidden, 32) == RD_OK;
+                if (s->q_maps_ok) s->attn_path = 3;
+            }
         }
         if (m->tc_ok) {
             // scratch for the partial sums: the largest need over the model's GEMM shapes and over
@@ -606,9 +629,10 @@ extern "C" int rd_set_gemm_path(rd_session* s, int32_t path) {
 }
 
 extern "C" int rd_set_attention_path(rd_session* s, int32_t path) {
-    if (!s || path < 0 || path > 2) return RD_E_INVALID_ARG;
+    if (!s || path < 0 || path > 3) return RD_E_INVALID_ARG;
     if (path >= 1 && !s->attn_capable) return RD_E_STATE;             // no tensor-core attention for this model
-    if (path == 2 && !s->att_maps_ok) return RD_E_STATE;
+    if (path >= 2 && !s->att_maps_ok) return RD_E_STATE;
+    if (path == 3 && !s->q_maps_ok) return RD_E_STATE;
     s->attn_path = path;
     return RD_OK;
 }
@@ -747,7 +771,7 @@ template <typename T> struct Eng {
         // K/V through the TMA ring for groups of more than 8 rows; smaller groups (the sequential decoder's
         // one row per sequence) do so little arithmetic per tile that the copies' latency is exposed, and the
         // cp.async kernel, whose loads every thread issues, is faster there (110.6 against 98.4 tok/s at 8k keys)
-        if (s->attn_path == 2 && s->grp_rows > ATT_TMA_MIN_ROWS) {
+        if (s->attn_path >= 2 && s->grp_rows > ATT_TMA_MIN_ROWS) {
             // Kc points at this layer inside block s->att_blk
             const int row_base = s->att_layer * s->sc.batch * c.n_heads * s->sc.max_context;
             LAUNCH_CLUSTER(s, (attn_tma_kernel<D, KW, NW>), (ns, c.n_heads, groups), 32 * NW, (AttTmaCfg<D, NW>::SMEM), ns,
@@ -764,6 +788,17 @@ template <typename T> struct Eng {
     static int attn_windowed_k(rd_session* s, const bf16* Kc, const bf16* Vc, int n_rows) {
         // groups of at most 32 rows: every warp takes half of a key tile, so all four warps work;
         // up to 64 rows: four warps of 16 queries; up to 128 rows: eight
+        if (s->attn_path == 3 && s->grp_rows == ATC_Q && !s->att_index && s->att_groups == 0) {
+            // prefill: 128 consecutive prompt rows per group, both products on tcgen05
+            const rd_config& c = s->m->cfg;
+            AtcMaps maps;
+            maps.q64 = s->q_map64; maps.q32 = s->q_map32; maps.kv = s->att_maps[s->att_blk];
+            const int row_base = s->att_layer * s->sc.batch * c.n_heads * s->sc.max_context;
+            const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
+            LAUNCH(s, attn_prefill_tc_kernel<D>, dim3(c.n_heads, (n_rows + ATC_Q - 1) / ATC_Q), ATC_THREADS, (AtcCfg<D>::SMEM), maps,
+                   s->row_pos, s->row_seq, n_rows, row_base, c.n_heads, s->sc.max_context, c.hidden, scale_log2, (bf16*)s->act_h, s->status);
+            return RD_OK;
+        }
         if (s->grp_rows <= 32) return attn_windowed_d<D, 32, 4>(s, Kc, Vc, n_rows);
         if (s->grp_rows <= 64) return attn_windowed_d<D, 64, 4>(s, Kc, Vc, n_rows);
         return attn_windowed_d<D, 64, 8>(s, Kc, Vc, n_rows);

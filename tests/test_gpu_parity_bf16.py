@@ -280,3 +280,28 @@ def test_attention_paths_agree_bit_for_bit(W, batch, L):
     for a, b in zip(*outs):
         assert np.array_equal(a, b)
     gm.close()
+
+
+@pytest.mark.parametrize("L", [100, 300, 700])
+def test_prefill_attention_on_tcgen05_agrees_with_the_mma_sync_kernel(L):
+    """Prefill attends 128-row groups with both products on tcgen05 (default; in lock step with the oracle
+    wherever a test prefills a bf16 model) or with the windowed mma.sync kernel (path 2).  Same inputs,
+    same bf16 rounding of P, different summation order: cache rows agree to bf16 rounding and the tokens
+    of a short generation are the same.  Prompts of one, three and six groups, the last one ragged."""
+    shape = rd_inputs.TWIN
+    w = rd_inputs.make_weights(**rd_inputs.shape_args(shape), seed=21, bf16=True, adapter_s_scale=0.25)
+    gm = gpu_model(shape, w, bf16=True)
+    outs = []
+    for path in (2, 3):
+        sess = rd.Session(gm, batch=1, max_context=L + 64, max_window=4, max_new_tokens=8, seed=13)
+        sess.set_attention_path(path)
+        sess.prefill(0, rd_inputs.make_prompt(L, shape["vocab"], seed=30), 2)
+        kv = [sess.read_kv(blk, l, which, 0, 0, L - 1) for blk, l in ((0, 1), (1, 0), (1, 3), (2, 1)) for which in (0, 1)]
+        for _ in range(6):
+            sess.df_step(4, 1, 0.0)
+        outs.append((kv, sess.tokens(0).copy()))
+        sess.close()
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert np.abs(a).max() > 0 and TOL.excess(b, a) <= 0 and np.sqrt(np.mean((a - b) ** 2)) < 5e-3
+    assert np.array_equal(outs[0][1], outs[1][1])
+    gm.close()

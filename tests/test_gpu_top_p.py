@@ -86,7 +86,9 @@ def test_bf16_twin_ragged_batch_top_p():
     """bf16 configuration (tensor-core GEMMs), ragged batch, adaptive exit, T = 1, top-p 0.9.  The
     logit tolerance moves the cumulative masses near the cut by a few percent: band 0.1."""
     shape = rd_inputs.TWIN
-    sess, sm = _pair(shape, 8, 16, 1.0, 0.9, batch=4, bf16=True, std=0.02)
+    # (the contractive adapter of the other bf16 tests: a row takes up to 16 recurrences here, along which
+    # rounding differences between two bf16 evaluations grow with the plain init)
+    sess, sm = _pair(shape, 8, 16, 1.0, 0.9, batch=4, bf16=True, std=0.02, adapter_s_scale=0.25)
     seqs = _prefill(sm, sess, shape, [5, 33, 12, 40], 4, 16)
     ls = LockStep(sm, sess, seqs, Tolerance(5e-2, 2e-2), tie_gap=3e-2, nucleus_band=0.1)
     for _ in range(40):
