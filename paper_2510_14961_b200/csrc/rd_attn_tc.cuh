@@ -11,8 +11,13 @@
 //   warp 0 / lane 0   TMA producer: Q once, then K and V tiles through a ring of stages
 //   warp 1 / lane 0   issues the MMAs; tcgen05.commit signals the softmax warps and frees stages
 //   warps 2-5         one query row per thread (TMEM lane = row): S from TMEM, causal mask, online
-//                     softmax in float32 (log2 domain), P to shared memory in the 128-byte swizzle,
-//                     then the tile's P V from TMEM into the running output in registers
+//                     softmax in float32 (log2 domain), P to shared memory in the 128-byte swizzle
+// O stays in TMEM and accumulates over the tiles.  A row's running maximum is only moved when a tile's
+// maximum exceeds it by more than 2^8 (P = 2^(s - m) then stays below 256, exact enough in bf16 and
+// float32, and the final O / l does not depend on which m was used); when it moves, the row's O is
+// rescaled in place (tcgen05.ld / st by the row's own thread, before it releases P: by then every MMA
+// issued before this tile's S has completed, the previous P V among them).  So a tile costs two
+// hand-offs (S ready, P ready) instead of four.
 // Q, K, V sub-tiles are the ones of rd_attn.cuh (64 columns with the 128-byte swizzle, 32 with the
 // 64-byte swizzle for the last third of a 96-wide head), written by TMA and described to the MMA by
 // shared-memory descriptors.  Every wait is bounded; on time-out the kernel raises the status word,
@@ -41,6 +46,17 @@ __device__ __forceinline__ uint64_t umma_desc_mn64(uint32_t saddr) {
 }
 // instruction descriptor with B given MN-major (bit 16)
 __host__ __device__ constexpr uint32_t umma_idesc_bmn(int bn) { return umma_idesc(bn) | (1u << 16); }
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 
 template <int D> struct AtcCfg {
     using T = AttTile<D>;
@@ -178,7 +194,6 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
             for (int t = 0; t < nt && ok; t++) {
                 const int s = t % S;
                 if (*abort_flag || !mbar_wait(p_full, t & 1)) { ok = false; break; }          // P(t) in shared memory, S free
-                if (t > 0 && !mbar_wait(o_free, (t - 1) & 1)) { ok = false; break; }          // O(t-1) read out of TMEM
                 tc_fence_after();
                 const uint32_t v0 = smem_u32(ring + s * C::KV_STAGE + T::BYTES);
 #pragma unroll
@@ -186,18 +201,19 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
 #pragma unroll
                     for (int k = 0; k < 4; k++)          // 16 keys per MMA: 16 rows of the V sub-tile further on
                         umma_bf16(tmem_base + (uint32_t)(C::O_COL + a * 64), umma_desc_k128(p0) + (uint64_t)(k * 2),
-                                  umma_desc_mn128(v0 + a * T::A_BYTES + k * 2048), idesc_o64, k ? 1u : 0u);
+                                  umma_desc_mn128(v0 + a * T::A_BYTES + k * 2048), idesc_o64, (t | k) ? 1u : 0u);
                 if (T::NB) {
 #pragma unroll
                     for (int k = 0; k < 4; k++)
                         umma_bf16(tmem_base + (uint32_t)(C::O_COL + T::NA * 64), umma_desc_k128(p0) + (uint64_t)(k * 2),
-                                  umma_desc_mn64(v0 + T::NA * T::A_BYTES + k * 1024), idesc_o32, k ? 1u : 0u);
+                                  umma_desc_mn64(v0 + T::NA * T::A_BYTES + k * 1024), idesc_o32, (t | k) ? 1u : 0u);
                 }
                 umma_commit(&kv_empty[s]);               // K and V of this stage have been read
-                umma_commit(o_full);
                 if (t + 1 < nt) {
                     if (*abort_flag || !mbar_wait(&kv_full[(t + 1) % S], ((t + 1) / S) & 1)) { ok = false; break; }
-                    issue_qk(t + 1);                     // runs while the softmax warps take O(t)
+                    issue_qk(t + 1);                     // its commit also covers the P V just issued
+                } else {
+                    umma_commit(o_full);                 // the last P V: O is complete
                 }
             }
             if (!ok) *abort_flag = 1;
@@ -207,10 +223,7 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
         const int quad = warp & 3;
         const int row = quad * 32 + lane;                 // row of the group = TMEM lane
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
-        float m = -INFINITY, l = 0.f;
-        float o[D];
-#pragma unroll
-        for (int j = 0; j < D; j++) o[j] = 0.f;
+        float m = -INFINITY, l = 0.f;                  // m: the maximum the row's P and O are scaled by (log2 domain)
         bool ok = true;
         for (int t = 0; t < nt && ok; t++) {
             if (*abort_flag || !mbar_wait(s_full, t & 1)) { ok = false; break; }
@@ -226,10 +239,25 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
                 sr[j] = __float_as_uint(v);
                 mx = fmaxf(mx, v);
             }
-            const float mn = fmaxf(m, mx);
-            const float u = mn == -INFINITY ? 0.f : mn;
-            const float corr = exp2f(m - u);
-            m = mn;
+            // move the row's maximum only when the tile exceeds it by more than 8 (a factor 256)
+            const bool move = mx > m + 8.0f || (m == -INFINITY && mx > -INFINITY);
+            if (__any_sync(0xffffffffu, move && t > 0 && l > 0.f)) {
+                // rescale O in place: every MMA before this tile's S has completed, so O is at rest
+                const float corr = move ? exp2f(m - mx) : 1.0f;       // (m = -inf: the row has nothing yet, corr 0 is harmless)
+#pragma unroll
+                for (int c = 0; c < D; c += 32) {
+                    uint32_t orow[32];
+                    tmem_ld32(t_lane + (uint32_t)(C::O_COL + c), orow);
+#pragma unroll
+                    for (int j = 0; j < 32; j++) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * corr);
+                    tmem_st32(t_lane + (uint32_t)(C::O_COL + c), orow);
+                }
+                if (move) l *= corr;
+            } else if (move) {
+                l *= (m == -INFINITY ? 0.f : exp2f(m - mx));
+            }
+            if (move) m = mx;
+            const float u = m == -INFINITY ? 0.f : m;
             float sum = 0.f;
             // P row: 64 bf16 = 8 chunks of 16 bytes, chunk c at (c ^ (row & 7)) of the row's 128 bytes
             uint8_t* prow = Ps + row * 128;
@@ -244,21 +272,22 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
                 }
                 *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            l = l * corr + sum;
+            l += sum;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // P visible to the tensor core's reads
             tc_fence_before();
             mbar_arrive(p_full);
-            if (!mbar_wait(o_full, t & 1)) { ok = false; break; }
+        }
+        float o[D];
+        if (ok && nt > 0 && !mbar_wait(o_full, 0)) ok = false;
+        if (ok) {
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D; c += 32) {
                 uint32_t orow[32];
                 tmem_ld32(t_lane + (uint32_t)(C::O_COL + c), orow);
 #pragma unroll
-                for (int j = 0; j < 32; j++) o[c + j] = o[c + j] * corr + __uint_as_float(orow[j]);
+                for (int j = 0; j < 32; j++) o[c + j] = __uint_as_float(orow[j]);
             }
-            tc_fence_before();
-            mbar_arrive(o_free);
         }
         if (!ok) *abort_flag = 1;
         if (ok && my_pos >= 0) {
