@@ -94,13 +94,14 @@ def test_batch_ragged_prompts_and_single_token_prompt():
 
 
 def test_prefill_longer_than_one_chunk_and_kv_cache_contents():
-    """A prompt longer than the 128-row prefill chunk; cache rows compared directly."""
-    model, gm, sess, sm = _setup(SMALL, 0, 4, 2, std=0.08, gain_jitter=0.1, max_ctx=320)
-    seqs = _prefill_both(sm, sess, SMALL, [300], 2, 4)
+    """A prompt longer than the 512-row prefill chunk (two chunks: 512 + 87 rows); cache rows compared
+    directly, across the chunk boundary too."""
+    model, gm, sess, sm = _setup(SMALL, 0, 4, 2, std=0.08, gain_jitter=0.1, max_ctx=640)
+    seqs = _prefill_both(sm, sess, SMALL, [600], 2, 4)
     for blk, name in enumerate(("prelude", "core", "coda")):
         for which, arr in ((0, seqs[0].caches[name].K), (1, seqs[0].caches[name].V)):
-            got = sess.read_kv(blk, 0, which, 0, 0, 299)
-            want = arr[0, :299].reshape(299, -1)
+            got = sess.read_kv(blk, 0, which, 0, 0, 599)
+            want = arr[0, :599].reshape(599, -1)
             assert np.abs(got - want).max() < 1e-4
     ls = LockStep(sm, sess, seqs, TOL)
     while not ls.all_done():
