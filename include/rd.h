@@ -155,6 +155,30 @@ void rd_session_destroy(rd_session* s);
  * next step.  Errors: INVALID_ARG, CAPACITY (n_prompt + max_new_tokens > max_context), CUDA. */
 int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r);
 
+/* rd_prefill_sliced -- admission of a sequence into a running batch (Appendix, "Larger Batch Sizes":
+ * new requests join between the steps of the sequences already decoding).  The result is that of
+ * rd_prefill, bit for bit (same kernels on the same chunks in the same order), but the work is cut
+ * into units -- one pass of P, R or the coda layers over one chunk of prompt rows (a chunk holds
+ * max(512, decode rows of the session) rows, rounded up to a multiple of 16) -- and the steps that
+ * follow work it off: each rd_df_step / rd_ar_step first enqueues `units_per_step` units
+ * (rd_set_prefill_units; default 1) of the oldest pending job, so the running sequences are held
+ * up by one unit per step instead of a whole prefill.  Until its last unit has
+ * been enqueued, sequence `seq` is stopped: it has no in-flight rows, a step does nothing for it,
+ * rd_committed / rd_poll_end report it as not done and leave it out of the seq = -1 totals (ask
+ * rd_prefill_pending whether admissions are still under way).  The step whose units finish the job
+ * is the first one the sequence takes part in.
+ * The prompt is copied before the call returns; nothing is allocated.  Jobs are worked off in the
+ * order of their registration.  A step called while no sequence is running only works on the jobs.
+ * Errors: those of rd_prefill; STATE if `seq` already has a pending job.  While a job is pending
+ * rd_prefill returns STATE (one prefill workspace per session).
+ * rd_prefill_advance enqueues up to `units` units right away (no decode step), rd_prefill_pending
+ * returns the number of jobs not yet finished (>= 0, or INVALID_ARG), rd_set_prefill_units sets the
+ * units a step works off (0: steps leave the jobs to rd_prefill_advance). */
+int rd_prefill_sliced(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r);
+int rd_prefill_advance(rd_session* s, int32_t units);
+int rd_prefill_pending(const rd_session* s);
+int rd_set_prefill_units(rd_session* s, int32_t units_per_step);
+
 /* rd_ar_step -- one token on every live sequence by the sequential recurrence (Section 3.1):
  * e = P(newest token), s_0, r applications of R, p = C(s_r), sample, commit.
  * Errors: STATE (a sequence is not prefetched, or a wavefront wider than one is open). */

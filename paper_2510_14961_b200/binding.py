@@ -19,7 +19,8 @@ EXPORTS = ["rd_load", "rd_free", "rd_session_create", "rd_session_destroy", "rd_
            "rd_debug_force_tokens", "rd_debug_read_kv", "rd_stats", "rd_set_gemm_path", "rd_strerror",
            "rd_last_cuda_error", "rd_profile_enable", "rd_profile_read", "rd_debug_read_kv_noalloc", "rd_set_launch_chaining",
            "rd_debug_expire_next_wait", "rd_set_fused_swiglu", "rd_set_attention_path", "rd_poll_begin", "rd_poll_end",
-           "rd_debug_gemm_sequence"]
+           "rd_debug_gemm_sequence", "rd_prefill_sliced", "rd_prefill_advance", "rd_prefill_pending",
+           "rd_set_prefill_units"]
 
 
 class RdConfig(C.Structure):
@@ -71,6 +72,10 @@ def lib():
         L.rd_session_destroy.argtypes = [vp]
         L.rd_session_destroy.restype = None
         L.rd_prefill.argtypes = [vp, i32, vp, i32, i32]
+        L.rd_prefill_sliced.argtypes = [vp, i32, vp, i32, i32]
+        L.rd_prefill_advance.argtypes = [vp, i32]
+        L.rd_prefill_pending.argtypes = [vp]
+        L.rd_set_prefill_units.argtypes = [vp, i32]
         L.rd_ar_step.argtypes = [vp, i32]
         L.rd_df_step.argtypes = [vp, i32, i32, f32]
         L.rd_sync.argtypes = [vp]
@@ -172,6 +177,22 @@ class Session:
     def prefill(self, seq, prompt, r):
         p = np.ascontiguousarray(prompt, dtype=np.int32)
         _check(lib().rd_prefill(self.handle, seq, p.ctypes.data, len(p), r), "rd_prefill")
+
+    def prefill_sliced(self, seq, prompt, r):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        _check(lib().rd_prefill_sliced(self.handle, seq, p.ctypes.data, len(p), r), "rd_prefill_sliced")
+
+    def prefill_advance(self, units):
+        _check(lib().rd_prefill_advance(self.handle, units), "rd_prefill_advance")
+
+    def prefill_pending(self):
+        n = lib().rd_prefill_pending(self.handle)
+        if n < 0:
+            _check(n, "rd_prefill_pending")
+        return n
+
+    def set_prefill_units(self, units_per_step):
+        _check(lib().rd_set_prefill_units(self.handle, units_per_step), "rd_set_prefill_units")
 
     def ar_step(self, r):
         _check(lib().rd_ar_step(self.handle, r), "rd_ar_step")

@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <deque>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -272,6 +273,9 @@ struct rd_session {
     int* prompt_stage[PROMPT_STAGES] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t prompt_ev[PROMPT_STAGES] = {nullptr, nullptr, nullptr, nullptr};
     int stage_next = 0;
+    struct PrefillJob { int seq, L, r, pass, c0; };
+    std::deque<PrefillJob> jobs;              // sliced prefills (rd_prefill_sliced), oldest first
+    int units_per_step = 1;                   // prefill units a step works off before its own kernels
     bool expire_next_wait = false;            // test aid: see rd_debug_expire_next_wait
     float* acc = nullptr;          // output of the plain GEMM kernel, [rows, n_out]
     size_t acc_elems = 0;
@@ -1007,33 +1011,83 @@ template <typename T> struct Eng {
         return gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)s->m->head, &s->m->t_head, h, c.vocab, n_rows, &acc);
     }
 
-    static int prefill_passes(rd_session* s, int seq, int n, int r, float* e_all, float* s_all) {
+    // One unit of a prefill: pass `pass` of the chunk of prompt rows that starts at c0.
+    // pass 0: P and s_0; passes 1..r: one simultaneous application of R; pass r+1: coda layers (fills
+    // the coda cache; no head).  Units must run pass by pass, chunk by chunk: pass i of a row attends
+    // the pass-i K/V of the rows before it.
+    static int prefill_unit(rd_session* s, int seq, int n, int r, int pass, int c0, float* e_all, float* s_all) {
         const rd_config& c = s->m->cfg;
         const int h = c.hidden;
-        for (int pass = 0; pass < r + 2; pass++) {
-            // pass 0: P and s_0 for every chunk; passes 1..r: one simultaneous application of R;
-            // pass r+1: coda layers (fills the coda cache; no head).
-            for (int c0 = 0; c0 < n; c0 += s->R) {
-                const int nr = std::min(s->R, n - c0);
-                s->grp_rows = ATT_QMAX;
-                s->att_index = nullptr;
-                s->att_groups = 0;
-                s->ctx_max = c0 + nr;
-                s->ctx_total = c0 + nr;
-                s->grp_ctx.clear();
-                for (int g0 = 0; g0 < nr; g0 += ATT_QMAX) s->grp_ctx.push_back(c0 + std::min(nr, g0 + ATT_QMAX));
-                LAUNCH(s, fill_rows_kernel, (s->R + 127) / 128, 128, 0, seq, c0, nr, s->R, s->row_pos, s->row_seq);
-                float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
-                float* zc = s_all + (size_t)c0 * h;
-                if (pass == 0) {
-                    RD_TRY(prelude(s, nr, ec));
-                    LAUNCH(s, init_state_kernel, dim3(nr, init_parts(h)), 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
-                           s->sc.seed, zc, (size_t)h, (float*)nullptr, 0.f, 1);
-                } else if (pass <= r) {
-                    RD_TRY(core(s, ec, zc, zc, nr));
-                } else {
-                    RD_TRY(coda(s, zc, nr, false));
-                }
+        const int nr = std::min(s->R, n - c0);
+        s->grp_rows = ATT_QMAX;
+        s->att_index = nullptr;
+        s->att_groups = 0;
+        s->ctx_max = c0 + nr;
+        s->ctx_total = c0 + nr;
+        s->grp_ctx.clear();
+        for (int g0 = 0; g0 < nr; g0 += ATT_QMAX) s->grp_ctx.push_back(c0 + std::min(nr, g0 + ATT_QMAX));
+        LAUNCH(s, fill_rows_kernel, (s->R + 127) / 128, 128, 0, seq, c0, nr, s->R, s->row_pos, s->row_seq);
+        float* ec = e_all + (size_t)c0 * h;    // this chunk's rows of e and of the latent
+        float* zc = s_all + (size_t)c0 * h;
+        if (pass == 0) {
+            RD_TRY(prelude(s, nr, ec));
+            LAUNCH(s, init_state_kernel, dim3(nr, init_parts(h)), 128, 0, s->row_pos, s->row_seq, s->row_steps, 0, h, c.init_sigma,
+                   s->sc.seed, zc, (size_t)h, (float*)nullptr, 0.f, 1);
+            return RD_OK;
+        }
+        if (pass <= r) return core(s, ec, zc, zc, nr);
+        return coda(s, zc, nr, false);
+    }
+
+    static int prefill_passes(rd_session* s, int seq, int n, int r, float* e_all, float* s_all) {
+        for (int pass = 0; pass < r + 2; pass++)
+            for (int c0 = 0; c0 < n; c0 += s->R) RD_TRY(prefill_unit(s, seq, n, r, pass, c0, e_all, s_all));
+        return RD_OK;
+    }
+
+    // Upload of a prompt through one of the session's pinned copies (the caller's buffer is only borrowed).
+    static int upload_prompt(rd_session* s, int seq, const int32_t* prompt, int L) {
+        const int buf = s->stage_next;
+        CU(cudaEventSynchronize(s->prompt_ev[buf]));      // the upload that last used this copy has finished
+        memcpy(s->prompt_stage[buf], prompt, (size_t)L * sizeof(int));
+        CU(cudaMemcpyAsync(s->tokens + (size_t)seq * s->tok_stride, s->prompt_stage[buf], (size_t)L * sizeof(int),
+                           cudaMemcpyHostToDevice, s->stream));
+        CU(cudaEventRecord(s->prompt_ev[buf], s->stream));
+        s->stage_next = (buf + 1) % rd_session::PROMPT_STAGES;
+        return RD_OK;
+    }
+
+    // Sequence state behind a prefill: |y_frozen| = L and one fresh in-flight row at position L-1
+    // (stop = true: the sequence is taken out of the steps instead, e.g. while its prompt is prefilled in slices).
+    static int start_sequence(rd_session* s, int seq, int L, bool stop) {
+        SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
+        const int is_done = (stop || s->sc.max_new_tokens <= 0) ? 1 : 0;
+        if (s->pooled) {
+            LAUNCH(s, seq_start_pool_kernel, 1, 32, 0, st, seq, L, s->sc.max_window, is_done, s->pool);
+            return RD_OK;
+        }
+        const int slot = seq * s->sc.max_window + (L - 1) % s->sc.max_window;
+        LAUNCH(s, seq_start_kernel, 1, 32, 0, st, seq, L, slot, is_done);
+        return RD_OK;
+    }
+
+    // Work on the sliced prefills (rd_prefill_sliced): up to `units` units of the oldest job; a job that
+    // finishes starts its sequence.
+    static int advance_jobs(rd_session* s, int units) {
+        while (units > 0 && !s->jobs.empty()) {
+            rd_session::PrefillJob& j = s->jobs.front();
+            const int n = j.L - 1;
+            if (n > 0 && j.pass < j.r + 2) {
+                RD_TRY(prefill_unit(s, j.seq, n, j.r, j.pass, j.c0, s->pf_e, s->pf_s));
+                units--;
+                j.c0 += s->R;
+                if (j.c0 >= n) { j.c0 = 0; j.pass++; }
+            }
+            if (n <= 0 || j.pass >= j.r + 2) {
+                RD_TRY(start_sequence(s, j.seq, j.L, false));
+                s->prefilled[j.seq] = 1; s->wave_open[j.seq] = 0;
+                s->host_prompt_len[j.seq] = j.L; s->host_steps[j.seq] = 0;
+                s->jobs.pop_front();
             }
         }
         return RD_OK;
@@ -1043,23 +1097,18 @@ template <typename T> struct Eng {
     // copy of its own, e and the latents of the prompt rows live in the session's workspace, and the
     // sequence's state is set by a kernel behind the passes.
     static int prefill(rd_session* s, int seq, const int32_t* prompt, int L, int r) {
-        const int buf = s->stage_next;
-        CU(cudaEventSynchronize(s->prompt_ev[buf]));      // the upload that last used this copy has finished
-        memcpy(s->prompt_stage[buf], prompt, (size_t)L * sizeof(int));
-        CU(cudaMemcpyAsync(s->tokens + (size_t)seq * s->tok_stride, s->prompt_stage[buf], (size_t)L * sizeof(int),
-                           cudaMemcpyHostToDevice, s->stream));
-        CU(cudaEventRecord(s->prompt_ev[buf], s->stream));
-        s->stage_next = (buf + 1) % rd_session::PROMPT_STAGES;
+        RD_TRY(upload_prompt(s, seq, prompt, L));
         const int n = L - 1;   // rows 0..L-2 are prefilled; L-1 is the first in-flight row
         if (n > 0) RD_TRY(prefill_passes(s, seq, n, r, s->pf_e, s->pf_s));
-        // sequence state: |y_frozen| = L, one fresh in-flight row at position L-1
-        SeqState st{s->n_prompt, s->n_committed, s->win_len, s->done, s->row_steps, s->row_iters, s->counters};
-        if (s->pooled) {
-            LAUNCH(s, seq_start_pool_kernel, 1, 32, 0, st, seq, L, s->sc.max_window, s->sc.max_new_tokens <= 0 ? 1 : 0, s->pool);
-            return RD_OK;
-        }
-        const int slot = seq * s->sc.max_window + (L - 1) % s->sc.max_window;
-        LAUNCH(s, seq_start_kernel, 1, 32, 0, st, seq, L, slot, s->sc.max_new_tokens <= 0 ? 1 : 0);
+        return start_sequence(s, seq, L, false);
+    }
+
+    // rd_prefill_sliced: the prompt is uploaded and the sequence taken out of the steps now; the passes are
+    // worked off by the steps that follow.
+    static int prefill_sliced(rd_session* s, int seq, const int32_t* prompt, int L, int r) {
+        RD_TRY(upload_prompt(s, seq, prompt, L));
+        RD_TRY(start_sequence(s, seq, L, true));
+        s->jobs.push_back(rd_session::PrefillJob{seq, L, r, 0, 0});
         return RD_OK;
     }
 };
@@ -1072,11 +1121,17 @@ static bool any_prefilled(const rd_session* s) {
     return false;
 }
 
-extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r) {
+static int prefill_args(const rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r) {
     if (!s || !prompt || seq < 0 || seq >= s->sc.batch || n_prompt < 1 || r < 0) return RD_E_INVALID_ARG;
     if ((long long)n_prompt + s->sc.max_new_tokens > s->sc.max_context) return RD_E_CAPACITY;
     for (int i = 0; i < n_prompt; i++)
         if (prompt[i] < 0 || prompt[i] >= s->m->cfg.vocab) return RD_E_INVALID_ARG;
+    return RD_OK;
+}
+
+extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r) {
+    RD_TRY(prefill_args(s, seq, prompt, n_prompt, r));
+    if (!s->jobs.empty()) return RD_E_STATE;     // the prefill workspace belongs to the sliced jobs
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::prefill(s, seq, prompt, n_prompt, r)
                                               : Eng<float>::prefill(s, seq, prompt, n_prompt, r);
     s->enqueue_epoch++;
@@ -1087,11 +1142,42 @@ extern "C" int rd_prefill(rd_session* s, int32_t seq, const int32_t* prompt, int
     return rc;
 }
 
+extern "C" int rd_prefill_sliced(rd_session* s, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t r) {
+    RD_TRY(prefill_args(s, seq, prompt, n_prompt, r));
+    for (const rd_session::PrefillJob& j : s->jobs)
+        if (j.seq == seq) return RD_E_STATE;
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::prefill_sliced(s, seq, prompt, n_prompt, r)
+                                              : Eng<float>::prefill_sliced(s, seq, prompt, n_prompt, r);
+    s->enqueue_epoch++;
+    if (rc == RD_OK) { s->prefilled[seq] = 0; s->wave_open[seq] = 0; }
+    return rc;
+}
+
+extern "C" int rd_prefill_advance(rd_session* s, int32_t units) {
+    if (!s || units < 0) return RD_E_INVALID_ARG;
+    if (s->jobs.empty() || units == 0) return RD_OK;
+    const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::advance_jobs(s, units) : Eng<float>::advance_jobs(s, units);
+    s->enqueue_epoch++;
+    return rc;
+}
+
+extern "C" int rd_prefill_pending(const rd_session* s) {
+    return s ? (int)s->jobs.size() : RD_E_INVALID_ARG;
+}
+
+extern "C" int rd_set_prefill_units(rd_session* s, int32_t units_per_step) {
+    if (!s || units_per_step < 0) return RD_E_INVALID_ARG;
+    s->units_per_step = units_per_step;
+    return RD_OK;
+}
+
 extern "C" int rd_ar_step(rd_session* s, int32_t r) {
     if (!s || r < 1) return RD_E_INVALID_ARG;
-    if (!any_prefilled(s)) return RD_E_STATE;
+    if (!any_prefilled(s) && s->jobs.empty()) return RD_E_STATE;
     for (int b = 0; b < s->sc.batch; b++)
         if (s->prefilled[b] && s->wave_open[b]) return RD_E_STATE;
+    RD_TRY(rd_prefill_advance(s, s->units_per_step));
+    if (!any_prefilled(s)) return RD_OK;         // only prefill work was due
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, 1, r, 0.f, false) : Eng<float>::decode_step(s, 1, r, 0.f, false);
     s->enqueue_epoch++;
     if (rc == RD_OK) s->stats.ar_steps++;
@@ -1101,7 +1187,9 @@ extern "C" int rd_ar_step(rd_session* s, int32_t r) {
 extern "C" int rd_df_step(rd_session* s, int32_t window, int32_t inner_iters, float exit_threshold) {
     if (!s || window < 1 || inner_iters < 1 || exit_threshold != exit_threshold) return RD_E_INVALID_ARG;
     if (window > s->sc.max_window) return RD_E_CAPACITY;
-    if (!any_prefilled(s)) return RD_E_STATE;
+    if (!any_prefilled(s) && s->jobs.empty()) return RD_E_STATE;
+    RD_TRY(rd_prefill_advance(s, s->units_per_step));
+    if (!any_prefilled(s)) return RD_OK;         // only prefill work was due
     const int rc = s->m->cfg.dtype == RD_BF16 ? Eng<bf16>::decode_step(s, window, inner_iters, exit_threshold, true)
                                               : Eng<float>::decode_step(s, window, inner_iters, exit_threshold, true);
     s->enqueue_epoch++;
