@@ -246,6 +246,39 @@ def torch_weights(shape, bf16, device, seed=0, std=0.02):
     return out
 
 
+def admission_latency(rd, model, stream, shape, wl):
+    """Step latency seen by three running sequences while a fourth is admitted (Appendix, "Larger Batch
+    Sizes"), with the prompt prefilled in one piece (rd_prefill) and in slices (rd_prefill_sliced):
+    one CUDA-event pair per step, 20 steps before the admission and 60 after it."""
+    import torch
+    B, W, L, r = 4, wl["window"], wl["prompt"] if not isinstance(wl["prompt"], tuple) else wl["prompt"][1], wl["prefill_r"]
+    n_steps, at = 80, 20
+    N = 60 + n_steps + 2 * W
+    prompts = [rd_inputs.make_prompt(L, shape["vocab"], seed=117 + b) for b in range(B)]
+    out = {"running_sequences": B - 1, "admitted_prompt": L, "prefill_r": r, "window": W}
+    for mode in ("whole", "sliced"):
+        sess = rd.Session(model, batch=B, max_context=L + N + 8, max_window=W, max_iters_per_pos=64, max_new_tokens=N,
+                          seed=1, stream=stream.cuda_stream)
+        for b in range(B - 1):
+            sess.prefill(b, prompts[b], 1)
+        for _ in range(2 * W):
+            sess.df_step(W, wl["inner"], 0.0)
+        sess.sync()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        with torch.cuda.stream(stream):
+            evs[0].record(stream)
+            for i in range(n_steps):
+                if i == at:
+                    (sess.prefill if mode == "whole" else sess.prefill_sliced)(B - 1, prompts[B - 1], r)
+                sess.df_step(W, wl["inner"], 0.0)
+                evs[i + 1].record(stream)
+        sess.sync()
+        ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_steps)]
+        out[mode] = {"step_ms_before": sorted(ms[:at])[at // 2], "worst_step_ms": max(ms), "total_ms": sum(ms)}
+        sess.close()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -574,6 +607,8 @@ def run_ours(args):
         "gpu_launches": int(launches0), "tc_gemm_launches": int(tc_launches),
         "commit_hist": lib_stats["commit_hist"],
     }
+    if args.admission:
+        line["admission"] = admission_latency(rd, model, stream, shape, wl)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
     if world > 1:
@@ -696,6 +731,8 @@ def main():
     ap.add_argument("--unfused-swiglu", action="store_true", help="A/B: SwiGLU as a separate kernel")
     ap.add_argument("--attention-path", type=int, default=-1, help="A/B: 3 default (TMA ring; tcgen05 prefill), 2 without the tcgen05 prefill kernel, 1 cp.async, 0 SIMT")
     ap.add_argument("--unchained", action="store_true", help="A/B: no programmatic dependent launch")
+    ap.add_argument("--admission", action="store_true",
+                    help="also measure the step latency of running sequences while one more is admitted (whole vs sliced prefill)")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
     if args.impl == "reference":
