@@ -8,11 +8,14 @@
 // K-major with the 128-byte swizzle TMA writes; the accumulator D[feature, row] lives in TMEM
 // (128 lanes x BN columns, fp32, two buffers).
 //
-// Persistent stream-K schedule: the (feature tile, row tile, k-block) units are numbered tile by
-// tile (the row tiles of one feature tile next to each other, so that their common weight tiles are
-// streamed close together in time) and cut into one contiguous share per CTA (two CTAs per SM while the row tile is at most
-// 128 wide), so every SM streams the same number of weight bytes through long-lived rings whatever
-// n_out is.  A share is a list of segments (tile, k-block range):
+// Persistent stream-K schedule: the (row tile, feature tile, k-block) units are numbered tile by
+// tile, all feature tiles of the first row tile before those of the second, and cut into one
+// contiguous share per CTA (two CTAs per SM while the row tile is at most 128 wide), so every SM
+// streams the same number of weight bytes through long-lived rings whatever n_out is.  With two row tiles (prefill chunks) the CTA half a grid away therefore
+// streams the same weight tile at the same moment for the other row tile, and one of the two reads
+// hits L2; numbered with the row tiles of a feature tile next to each other, a CTA came back to a
+// weight tile a whole tile later, with more than an L2's worth of other weights streamed in between.
+// A share is a list of segments (tile, k-block range):
 //   warp 0 / lane 0   TMA producer: fills a ring of STAGES {A,B} stages, mbarrier complete_tx
 //   warp 1 / lane 0   issues tcgen05.mma (4 per stage, K = 16 each); tcgen05.commit frees the stage
 //                     and, at the end of a segment, publishes the accumulator buffer
@@ -311,7 +314,7 @@ template <int BN> struct TcCfg {
 
 struct TcParams {
     int kb;                    // k-blocks per tile
-    int n_tiles_n;             // row tiles; tile number = (feature tile / MT) * n_tiles_n + row tile
+    int n_tiles_m;             // feature tiles of a unit's width; tile number = row tile * n_tiles_m + feature tile / MT
     long long units;           // tiles * kb
     int per;                   // units per CTA
     int max_seg;               // scratch slots per CTA
@@ -368,14 +371,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], C::STAGE_BYTES);
-                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM * C::MT, &full[i]);
+                tma_load_2d(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM * C::MT, &full[i]);
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
                 if (i == skip) continue;
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
-                tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[i]);
+                tma_load_2d(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[i]);
             }
             int issued = pre;
             for (int i = pre; i < n_units; i++) {
@@ -385,8 +388,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 mbar_expect_tx(&full[s], C::STAGE_BYTES);
                 uint8_t* a = smem + s * C::STAGE_BYTES;
-                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile / p.n_tiles_n) * TC_BM * C::MT, &full[s]);
-                tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile % p.n_tiles_n) * BN, &full[s]);
+                tma_load_2d(a, &tmap_w, kblk * TC_BK, (tile % p.n_tiles_m) * TC_BM * C::MT, &full[s]);
+                tma_load_2d(a + C::A_BYTES, &tmap_x, kblk * TC_BK, (tile / p.n_tiles_m) * BN, &full[s]);
                 issued = i + 1;
             }
             if (*abort_flag) {
@@ -455,7 +458,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (p.fuse.act_out) {
                     // whole tile (ka == 0, len == kb): SwiGLU straight from the accumulator
                     const int tile = (int)(u / p.kb);
-                    const int ftu = tile / p.n_tiles_n, rt = tile % p.n_tiles_n;
+                    const int ftu = tile % p.n_tiles_m, rt = tile / p.n_tiles_m;
                     if constexpr (BN >= 32) {
 #pragma unroll 1
                         for (int c = 0; c < C::MT * BN; c += 32) {
@@ -505,19 +508,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     }
 }
 
-// Position of a unit in (feature tile [pair], row tile, k-block) order, advanced without division.
+// Position of a unit in (row tile, feature tile [pair], k-block) order, advanced without division.
 struct UnitCursor {
     int ft, rt, kblk;
-    __device__ UnitCursor(long long u, int kb, int n_tiles_n) {
+    __device__ UnitCursor(long long u, int kb, int n_tiles_m) {
         const long long tile = u / kb;
         kblk = (int)(u % kb);
-        ft = (int)(tile / n_tiles_n);
-        rt = (int)(tile % n_tiles_n);
+        ft = (int)(tile % n_tiles_m);
+        rt = (int)(tile / n_tiles_m);
     }
-    __device__ __forceinline__ void next(int kb, int n_tiles_n) {
+    __device__ __forceinline__ void next(int kb, int n_tiles_m) {
         if (++kblk == kb) {
             kblk = 0;
-            if (++rt == n_tiles_n) { rt = 0; ft++; }
+            if (++ft == n_tiles_m) { ft = 0; rt++; }
         }
     }
 };
@@ -590,18 +593,18 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 if (rank == 0) mbar_expect_tx(&full[i], 2 * C::STAGE_BYTES);
                 tma_load_2d_pair(smem + i * C::STAGE_BYTES, &tmap_w, kblk * TC_BK,
-                                 ((tile / p.n_tiles_n) * 2 + (int)rank) * TC_BM, map_to_rank(&full[i], 0));
+                                 ((tile % p.n_tiles_m) * 2 + (int)rank) * TC_BM, map_to_rank(&full[i], 0));
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kblk = (int)(u % p.kb);
                 tma_load_2d_pair(smem + i * C::STAGE_BYTES + C::A_BYTES, &tmap_x, kblk * TC_BK,
-                                 (tile % p.n_tiles_n) * C::BN + (int)rank * (C::BN / 2), map_to_rank(&full[i], 0));
+                                 (tile / p.n_tiles_m) * C::BN + (int)rank * (C::BN / 2), map_to_rank(&full[i], 0));
             }
             int issued = pre;
             // no division in this loop: it sets the pace of the pair (measured: 665 -> 320 cycles per unit)
-            UnitCursor cur(u0 + pre, p.kb, p.n_tiles_n);
+            UnitCursor cur(u0 + pre, p.kb, p.n_tiles_m);
             int s = pre % C::STAGES;
             uint32_t parity = (uint32_t)(((pre / C::STAGES) - 1) & 1);
             for (int i = pre; i < n_units; i++) {
@@ -612,7 +615,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 tma_load_2d_pair(a, &tmap_w, cur.kblk * TC_BK, (cur.ft * 2 + (int)rank) * TC_BM, bar);
                 tma_load_2d_pair(a + C::A_BYTES, &tmap_x, cur.kblk * TC_BK, cur.rt * C::BN + (int)rank * (C::BN / 2), bar);
                 issued = i + 1;
-                cur.next(p.kb, p.n_tiles_n);
+                cur.next(p.kb, p.n_tiles_m);
                 if (++s == C::STAGES) { s = 0; parity ^= 1; }
             }
             if (*abort_flag && rank == 0) {
@@ -681,7 +684,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_con
                 if (p.fuse.act_out) {
                     // whole tile: SwiGLU straight from this CTA's 128 features of the accumulator
                     const int tile = (int)(u / p.kb);
-                    const int ft = (tile / p.n_tiles_n) * 2 + (int)rank, rt = tile % p.n_tiles_n;
+                    const int ft = (tile % p.n_tiles_m) * 2 + (int)rank, rt = tile / p.n_tiles_m;
                     const int feat = (ft * TC_BM + quad * 32 + lane) >> 1;
 #pragma unroll 1
                     for (int c = 0; c < C::BN; c += 32) {
@@ -798,7 +801,7 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
     const TcPlan pl = tc_plan(K, n_out, n_rows, n_sms, pair, fuse != nullptr);
     if (!fuse && pl.scratch_elems > scratch_elems) return RD_E_INVALID_ARG;
     TcParams p;
-    p.kb = pl.kb; p.n_tiles_n = pl.n_tiles_n; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
+    p.kb = pl.kb; p.n_tiles_m = pl.n_tiles_m; p.units = pl.units; p.per = pl.per; p.max_seg = pl.max_seg;
     p.scratch = scratch; p.status = status;
     p.fuse = fuse ? *fuse : TcParamsFuse{nullptr, 0, 0, 0};
     p.spin_limit = TC_SPIN_LIMIT; p.skip_unit = -1;
@@ -808,7 +811,7 @@ static inline int tc_gemm(cudaStream_t st, const TcAct& ta, const TcWeight& tw, 
         p.spin_limit = 1u << 12; p.skip_unit = 0;
         *expire_wait = false;
     }
-    out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_n = pl.n_tiles_n; out->bn = pl.bn;
+    out->scratch = scratch; out->kb = pl.kb; out->per = pl.per; out->n_tiles_m = pl.n_tiles_m; out->bn = pl.bn;
     out->max_seg = pl.max_seg; out->mt_shift = pl.mt == 2 ? 1 : 0;
     switch (pl.bn_idx) {
         case 0: return tc_launch<16>(st, tw.map, ta.map[0], p, pl.grid, chained);

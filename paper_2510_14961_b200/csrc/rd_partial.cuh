@@ -10,12 +10,12 @@
 
 namespace rd {
 
-// Tile number = (feature tile >> mt_shift) * n_tiles_n + (row tile).  Units (tile, k-block) are numbered tile by
+// Tile number = (row tile) * n_tiles_m + (feature tile >> mt_shift).  Units (tile, k-block) are numbered tile by
 // tile, kb per tile; CTA g owns units [g*per, (g+1)*per).
 // The j-th tile CTA g touches went to slot g*max_seg + j, laid out [feature tile][bn rows][128 features].
 struct PartialSums {
     const float* scratch;
-    int kb, per, n_tiles_n, bn, max_seg;
+    int kb, per, n_tiles_m, bn, max_seg;
     int mt_shift;         // a tile covers 1 << mt_shift feature tiles of 128 (slot: [feature tile][bn rows][128])
 };
 
@@ -31,7 +31,7 @@ __device__ __forceinline__ float4 row_source_load4(const RowSource& s, int r, in
     const PartialSums& d = s.part;
     // (unit numbers stay far below 2^31: 32-bit arithmetic)
     const unsigned ft = (unsigned)(m >> 7);
-    const unsigned tile = (ft >> d.mt_shift) * d.n_tiles_n + (unsigned)(r / d.bn);
+    const unsigned tile = (unsigned)(r / d.bn) * d.n_tiles_m + (ft >> d.mt_shift);
     const unsigned t_lo = tile * (unsigned)d.kb;
     const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
     const size_t in_slot = ((size_t)(ft & ((1u << d.mt_shift) - 1)) * d.bn + (size_t)(r % d.bn)) * 128 + (m & 127);
@@ -97,7 +97,7 @@ __device__ __forceinline__ RowSlots<MAXQ> row_source_locate(const RowSource& s, 
     }
     const PartialSums& d = s.part;
     const unsigned ft = (unsigned)(m >> 7);
-    const unsigned tile = (ft >> d.mt_shift) * d.n_tiles_n + (unsigned)(r / d.bn);
+    const unsigned tile = (unsigned)(r / d.bn) * d.n_tiles_m + (ft >> d.mt_shift);
     const unsigned t_lo = tile * (unsigned)d.kb;
     const int g_lo = (int)(t_lo / (unsigned)d.per), g_hi = (int)((t_lo + d.kb - 1) / (unsigned)d.per);
     const size_t in_slot = ((size_t)(ft & ((1u << d.mt_shift) - 1)) * d.bn + (size_t)(r % d.bn)) * 128 + (m & 127);
