@@ -21,6 +21,17 @@ __device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+// four consecutive values as one store (dst aligned to four elements); same roundings as from_f
+__device__ __forceinline__ void store4(float* dst, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(bf16* dst, float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 w;
+    w.x = *reinterpret_cast<const uint32_t*>(&lo);
+    w.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst) = w;
+}
 
 // 16-byte vector load of 16/sizeof(T) elements, widened to float.
 template <typename T> struct Vec16;
@@ -204,7 +215,7 @@ __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restr
 // CL blocks per row: 8 while few rows are in flight (latency), 2 for 128 rows and more (one wave of
 // blocks, each thread several groups of four).
 template <typename TO, int CL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, CL == 2 ? 4 : 1)
 rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,
                size_t ldx, const float* __restrict__ g, int hidden, float eps, TO* __restrict__ out, size_t ldo,
                const int* __restrict__ row_pos) {
@@ -228,7 +239,10 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     const int m_first = m0 + threadIdx.x * 4;
     RowSlots<NQ> first_slots;
     first_slots.n = NQ + 1;
-    if (m_first < m1) first_slots = row_source_locate<NQ>(src, r, m_first);
+    // (many rows in flight, CL == 2: the kernel is bound by its instruction count and its registers,
+    // not by the latency after the wait; every group goes through row_source_load4)
+    if constexpr (CL > 2)
+        if (m_first < m1) first_slots = row_source_locate<NQ>(src, r, m_first);
     pdl_wait();
     cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
     if (row_pos && row_pos[r] < 0) return;                       // the whole cluster leaves
@@ -237,7 +251,9 @@ rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr,
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     float ss = 0.f;
     for (int m = m_first; m < m1; m += blockDim.x * 4) {
-        float4 v = (m == m_first && first_slots.n <= NQ) ? row_source_fetch<NQ>(first_slots) : row_source_load4(src, r, m);
+        float4 v;
+        if constexpr (CL > 2) v = (m == m_first && first_slots.n <= NQ) ? row_source_fetch<NQ>(first_slots) : row_source_load4(src, r, m);
+        else v = row_source_load4(src, r, m);
         if (resid) {
             const float4 q = *reinterpret_cast<const float4*>(resid + (size_t)r * ldr + m);
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
@@ -376,7 +392,9 @@ gemm_simt_kernel(const T* __restrict__ A, size_t lda, const T* __restrict__ W, i
 // Rotary embedding on adjacent pairs of q and k, then: q -> q_t (GEMM/attention input type),
 // k, v -> the row's own cache entry (overwrite: KV-cache sharing, Section 3.2).
 // src: result of the QKV GEMM, [rows, 3h] (q | k | v).  cos/sin: [max_ctx, d/2] float32.
-template <typename T>
+// LOCATE: the slots of the first group are worked out before the wait for the GEMM (few rows in flight:
+// latency); without it every group goes through row_source_load4 (many rows: instruction count).
+template <typename T, bool LOCATE>
 __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_pos,
                                const int* __restrict__ row_seq, const float* __restrict__ cos_t,
                                const float* __restrict__ sin_t, int hidden, int head_dim, T* __restrict__ q_t,
@@ -390,16 +408,18 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
     const int m_first = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
     RowSlots<NQ> sq, sk, sv;
     sq.n = NQ + 1;
-    if (m_first < hidden) {
-        sq = row_source_locate<NQ>(src, r, m_first);
-        sk = row_source_locate<NQ>(src, r, hidden + m_first);
-        sv = row_source_locate<NQ>(src, r, 2 * hidden + m_first);
-    }
+    if constexpr (LOCATE)
+        if (m_first < hidden) {
+            sq = row_source_locate<NQ>(src, r, m_first);
+            sk = row_source_locate<NQ>(src, r, hidden + m_first);
+            sv = row_source_locate<NQ>(src, r, 2 * hidden + m_first);
+        }
+    const bool vec = (head_dim & 3) == 0;      // a group of four stays inside one head: 8- or 16-byte stores
     pdl_wait();
     // four features = two rotary pairs per thread and turn
     for (int m = m_first; m < hidden; m += gridDim.y * blockDim.x * 4) {
         // the sums are requested first; the row's position (and with it the rotary angles) meanwhile
-        const bool located = m == m_first && sq.n <= NQ && sk.n <= NQ && sv.n <= NQ;
+        const bool located = LOCATE && m == m_first && sq.n <= NQ && sk.n <= NQ && sv.n <= NQ;
         const float4 q = located ? row_source_fetch<NQ>(sq) : row_source_load4(src, r, m),
                      k = located ? row_source_fetch<NQ>(sk) : row_source_load4(src, r, hidden + m),
                      v = located ? row_source_fetch<NQ>(sv) : row_source_load4(src, r, 2 * hidden + m);
@@ -411,12 +431,18 @@ __global__ void rope_kv_kernel(const RowSource src, const int* __restrict__ row_
         const int i0 = ((m % head_dim) >> 1), i1 = (((m + 2) % head_dim) >> 1);
         const float c0 = cos_t[(size_t)p * half + i0], s0 = sin_t[(size_t)p * half + i0];
         const float c1 = cos_t[(size_t)p * half + i1], s1 = sin_t[(size_t)p * half + i1];
+        // the two pairs may lie in different heads when head_dim is not a multiple of 4
+        const size_t d0 = (size_t)(m / head_dim) * head_stride + (m % head_dim);
+        if (vec) {
+            store4(qdst + m, q.x * c0 - q.y * s0, q.x * s0 + q.y * c0, q.z * c1 - q.w * s1, q.z * s1 + q.w * c1);
+            store4(kseq + d0, k.x * c0 - k.y * s0, k.x * s0 + k.y * c0, k.z * c1 - k.w * s1, k.z * s1 + k.w * c1);
+            store4(vseq + d0, v.x, v.y, v.z, v.w);
+            continue;
+        }
         qdst[m] = from_f<T>(q.x * c0 - q.y * s0);
         qdst[m + 1] = from_f<T>(q.x * s0 + q.y * c0);
         qdst[m + 2] = from_f<T>(q.z * c1 - q.w * s1);
         qdst[m + 3] = from_f<T>(q.z * s1 + q.w * c1);
-        // the two pairs may lie in different heads when head_dim is not a multiple of 4
-        const size_t d0 = (size_t)(m / head_dim) * head_stride + (m % head_dim);
         const size_t d1 = (size_t)((m + 2) / head_dim) * head_stride + ((m + 2) % head_dim);
         kseq[d0] = from_f<T>(k.x * c0 - k.y * s0);
         kseq[d0 + 1] = from_f<T>(k.x * s0 + k.y * c0);

@@ -361,7 +361,8 @@ template <typename T> static void want_max_carveout_typed() {
     want_max_carveout(gemm_simt_kernel<T, 1>);
     want_max_carveout(gemm_simt_kernel<T, 4>);
     want_max_carveout(gemm_simt_kernel<T, 8>);
-    want_max_carveout(rope_kv_kernel<T>);
+    want_max_carveout(rope_kv_kernel<T, true>);
+    want_max_carveout(rope_kv_kernel<T, false>);
     want_max_carveout(attn_row_kernel<T>);
     want_max_carveout(swiglu_kernel<T>);
 }
@@ -831,8 +832,13 @@ template <typename T> struct Eng {
         const float* x_in = lazy ? s->x : in.src.plain;
         RowSource acc;
         RD_TRY(gemm(s, (T*)s->act_h, h, &s->t_act_h, (T*)L.wqkv, &L.t_qkv, h, 3 * h, n_rows, &acc));
-        LAUNCH(s, rope_kv_kernel<T>, dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
-               (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
+        if (n_rows >= 128) {
+            LAUNCH(s, (rope_kv_kernel<T, false>), dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+                   (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
+        } else {
+            LAUNCH(s, (rope_kv_kernel<T, true>), dim3(n_rows, 16), 128, 0, acc, s->row_pos, s->row_seq, s->cos_t, s->sin_t, h, c.head_dim,
+                   (T*)s->q_t, Kc, Vc, s->seq_stride, s->head_stride);
+        }
         const int br = bracket_open(s, 1, s->ctx_total * 2 * h * sizeof(T));
         bool windowed = false;
         if constexpr (sizeof(T) == 2) {
