@@ -212,8 +212,8 @@ __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restr
 // through distributed shared memory (added in block order).  `src` is a finished array or the
 // partial sums of the GEMM before (added here, in k order); with x_store, x is written out as the
 // new residual stream (x_store may alias resid).
-// CL blocks per row: 8 while few rows are in flight (latency), 2 for 128 rows and more (one wave of
-// blocks, each thread several groups of four).
+// CL blocks per row: 8 up to 32 rows in flight (latency), 4 up to 127 rows and 2 from 128 rows on (as
+// few waves of blocks as possible, each thread several groups of four).
 template <typename TO, int CL>
 __global__ void __launch_bounds__(256, CL == 2 ? 4 : 1)
 rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,

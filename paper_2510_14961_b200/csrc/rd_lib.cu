@@ -356,6 +356,7 @@ template <typename F> static void want_max_carveout(F* kern) {
 template <typename T> static void want_max_carveout_typed() {
     want_max_carveout(embed_kernel<T>);
     want_max_carveout(rmsnorm_kernel<T, 8>);
+    want_max_carveout(rmsnorm_kernel<T, 4>);
     want_max_carveout(rmsnorm_kernel<T, 2>);
     want_max_carveout(concat_kernel<T>);
     want_max_carveout(gemm_simt_kernel<T, 1>);
@@ -742,6 +743,8 @@ template <typename T> struct Eng {
     static int norm(rd_session* s, const Pending& in, float* x_store, const float* g, TO* out, int n_rows) {
         const int h = s->m->cfg.hidden;
         if (n_rows >= 128) return norm_cl<TO, 2>(s, in, x_store, g, out, n_rows);   // (4-block clusters at 256 rows: no difference in an A/B)
+        // one wave of blocks: 8 x 64 blocks of 256 threads do not fit the GPU at once
+        if (n_rows > 32) return norm_cl<TO, 4>(s, in, x_store, g, out, n_rows);
         return norm_cl<TO, 8>(s, in, x_store, g, out, n_rows);
     }
     template <typename TO, int CL>
