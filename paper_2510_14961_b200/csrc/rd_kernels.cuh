@@ -215,7 +215,7 @@ __global__ void embed_kernel(const int* __restrict__ row_pos, const int* __restr
 // CL blocks per row: 8 up to 32 rows in flight (latency), 4 up to 127 rows and 2 from 128 rows on (as
 // few waves of blocks as possible, each thread several groups of four).
 template <typename TO, int CL>
-__global__ void __launch_bounds__(256, CL == 2 ? 4 : 1)
+__global__ void __launch_bounds__(256, CL == 2 ? 4 : 3)
 rmsnorm_kernel(const RowSource src, const float* __restrict__ resid, size_t ldr, float* __restrict__ x_store,
                size_t ldx, const float* __restrict__ g, int hidden, float eps, TO* __restrict__ out, size_t ldo,
                const int* __restrict__ row_pos) {
