@@ -8,16 +8,18 @@
 //   O[128 q, D]      += P V          A = P (bf16, written to shared memory by the softmax warps),
 //                                    B = V tile as it lies in the cache, [key][d] (MN-major), N = 64 (+ 32)
 // One CTA per (group of 128 rows, head), no key splits: a group's keys are walked tile by tile.
-//   warp 0 / lane 0   TMA producer: Q once, then K and V tiles through a ring of stages
+//   warp 0 / lane 0   TMA producer: Q once, then K and V tiles through rings of stages (K one tile ahead of V)
 //   warp 1 / lane 0   issues the MMAs; tcgen05.commit signals the softmax warps and frees stages
 //   warps 2-5         one query row per thread (TMEM lane = row): S from TMEM, causal mask, online
 //                     softmax in float32 (log2 domain), P to shared memory in the 128-byte swizzle
 // O stays in TMEM and accumulates over the tiles.  A row's running maximum is only moved when a tile's
 // maximum exceeds it by more than 2^8 (P = 2^(s - m) then stays below 256, exact enough in bf16 and
 // float32, and the final O / l does not depend on which m was used); when it moves, the row's O is
-// rescaled in place (tcgen05.ld / st by the row's own thread, before it releases P: by then every MMA
-// issued before this tile's S has completed, the previous P V among them).  So a tile costs two
-// hand-offs (S ready, P ready) instead of four.
+// rescaled in place (tcgen05.ld / st by the row's own thread, before it releases P).
+// S is double-buffered in TMEM and K has its own barriers: Q K^T of tile t + 2 is issued as soon as the
+// softmax warps have read S(t), so S(t + 1) is ready when they finish tile t and the tensor core works
+// under the softmax instead of in turn with it.  Before a softmax thread touches O (rescale) or the P
+// buffer for tile t it waits for the commit behind P V of tile t - 1 (the barrier that also frees that V tile).
 // Q, K, V sub-tiles are the ones of rd_attn.cuh (64 columns with the 128-byte swizzle, 32 with the
 // 64-byte swizzle for the last third of a 96-wide head), written by TMA and described to the MMA by
 // shared-memory descriptors.  Every wait is bounded; on time-out the kernel raises the status word,
@@ -47,6 +49,12 @@ __device__ __forceinline__ uint64_t umma_desc_mn64(uint32_t saddr) {
 // instruction descriptor with B given MN-major (bit 16)
 __host__ __device__ constexpr uint32_t umma_idesc_bmn(int bn) { return umma_idesc(bn) | (1u << 16); }
 
+// 2^x, one MUFU instruction (relative error 2^-22; -inf gives 0): P is rounded to bf16 right after
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
@@ -68,6 +76,7 @@ template <int D> struct AtcCfg {
     static constexpr int SMEM = 1024 + Q_BYTES + ATC_STAGES * KV_STAGE + P_BYTES + 256;
     static constexpr int TMEM_COLS = 256;                                     // S 64 | O 64 (+64) | O 32
     static constexpr int O_COL = 64;
+    static constexpr int S1_COL = 192;                                        // second S buffer
 };
 
 struct AtcMaps {
@@ -89,10 +98,12 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
     uint8_t* ring = Qs + C::Q_BYTES;
     uint8_t* Ps = ring + S * C::KV_STAGE;
     uint64_t* q_full = (uint64_t*)(Ps + C::P_BYTES);
-    uint64_t* kv_full = q_full + 1;           // [S]
-    uint64_t* kv_empty = kv_full + S;         // [S]
-    uint64_t* s_full = kv_empty + S;
-    uint64_t* p_full = s_full + 1;
+    uint64_t* k_full = q_full + 1;            // [S]  K tile of a stage landed
+    uint64_t* k_empty = k_full + S;           // [S]  ... has been read by its Q K^T
+    uint64_t* v_full = k_empty + S;           // [S]
+    uint64_t* v_empty = v_full + S;           // [S]  V tile read by its P V (also: that P V has completed)
+    uint64_t* s_full = v_empty + S;           // [2]  one per S buffer
+    uint64_t* p_full = s_full + 2;
     uint64_t* o_full = p_full + 1;
     uint64_t* o_free = o_full + 1;
     uint32_t* tmem_slot = (uint32_t*)(o_free + 1);
@@ -103,8 +114,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
     const int hd = blockIdx.x, r0 = blockIdx.y * ATC_Q;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < S; s++) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        mbar_init(s_full, 1); mbar_init(p_full, ATC_Q); mbar_init(o_full, 1); mbar_init(o_free, ATC_Q);
+        for (int s = 0; s < S; s++) {
+            mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+            mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+        }
+        mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1); mbar_init(p_full, 4); mbar_init(o_full, 1); mbar_init(o_free, ATC_Q);
         *abort_flag = 0;
         kv_len_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -139,28 +153,42 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
 #pragma unroll
             for (int a = 0; a < C::NA; a++) tma_load_2d(Qs + a * C::QA_BYTES, &maps.q64, hd * D + a * 64, r0, q_full);
             if (C::NB) tma_load_2d(Qs + C::NA * C::QA_BYTES, &maps.q32, hd * D + C::NA * 64, r0, q_full);
-            int issued = 0;
-            for (int t = 0; t < nt; t++) {
+            // K runs one tile ahead of V: the K tile of a stage is free as soon as its Q K^T has been
+            // issued and completed, the V tile only after the P V of the same keys
+            int issued_k = 0, issued_v = 0;
+            auto load_k = [&](int t) {
                 const int s = t % S;
-                if (t >= S && (*abort_flag || !mbar_wait(&kv_empty[s], ((t / S) - 1) & 1))) { *abort_flag = 1; break; }
                 uint8_t* kdst = ring + s * C::KV_STAGE;
-                uint8_t* vdst = kdst + T::BYTES;
                 const int y = head_row0 + t * ATT_KT;
-                mbar_expect_tx(&kv_full[s], C::KV_STAGE);
+                mbar_expect_tx(&k_full[s], T::BYTES);
 #pragma unroll
-                for (int a = 0; a < T::NA; a++) {
-                    tma_load_2d(kdst + a * T::A_BYTES, &maps.kv.k64, a * 64, y, &kv_full[s]);
-                    tma_load_2d(vdst + a * T::A_BYTES, &maps.kv.v64, a * 64, y, &kv_full[s]);
+                for (int a = 0; a < T::NA; a++) tma_load_2d(kdst + a * T::A_BYTES, &maps.kv.k64, a * 64, y, &k_full[s]);
+                if (T::NB) tma_load_2d(kdst + T::NA * T::A_BYTES, &maps.kv.k32, T::NA * 64, y, &k_full[s]);
+                issued_k = t + 1;
+            };
+            auto load_v = [&](int t) {
+                const int s = t % S;
+                uint8_t* vdst = ring + s * C::KV_STAGE + T::BYTES;
+                const int y = head_row0 + t * ATT_KT;
+                mbar_expect_tx(&v_full[s], T::BYTES);
+#pragma unroll
+                for (int a = 0; a < T::NA; a++) tma_load_2d(vdst + a * T::A_BYTES, &maps.kv.v64, a * 64, y, &v_full[s]);
+                if (T::NB) tma_load_2d(vdst + T::NA * T::A_BYTES, &maps.kv.v32, T::NA * 64, y, &v_full[s]);
+                issued_v = t + 1;
+            };
+            load_k(0);
+            for (int t = 0; t < nt; t++) {
+                if (t + 1 < nt) {
+                    if (t + 1 >= S && (*abort_flag || !mbar_wait(&k_empty[(t + 1) % S], (((t + 1) / S) - 1) & 1))) { *abort_flag = 1; break; }
+                    load_k(t + 1);
                 }
-                if (T::NB) {
-                    tma_load_2d(kdst + T::NA * T::A_BYTES, &maps.kv.k32, T::NA * 64, y, &kv_full[s]);
-                    tma_load_2d(vdst + T::NA * T::A_BYTES, &maps.kv.v32, T::NA * 64, y, &kv_full[s]);
-                }
-                issued = t + 1;
+                if (t >= S && (*abort_flag || !mbar_wait(&v_empty[t % S], ((t / S) - 1) & 1))) { *abort_flag = 1; break; }
+                load_v(t);
             }
             if (*abort_flag) {
                 mbar_wait(q_full, 0);
-                for (int t = max(0, issued - S); t < issued; t++) mbar_wait(&kv_full[t % S], (t / S) & 1);
+                for (int t = max(0, issued_k - S); t < issued_k; t++) mbar_wait(&k_full[t % S], (t / S) & 1);
+                for (int t = max(0, issued_v - S); t < issued_v; t++) mbar_wait(&v_full[t % S], (t / S) & 1);
             }
         }
     } else if (warp == 1) {
@@ -171,29 +199,36 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
             constexpr uint32_t idesc_o32 = umma_idesc_bmn(32);
             const uint32_t q0 = smem_u32(Qs), p0 = smem_u32(Ps);
             bool ok = mbar_wait(q_full, 0);
+            // S(t) goes to buffer t & 1 (columns 0..63 / S1_COL..): Q K^T of tile t + 2 is issued as soon as
+            // the softmax warps have read S(t), so they find S(t + 1) waiting when they are done with tile t
             auto issue_qk = [&](int t) {
                 const uint32_t k0 = smem_u32(ring + (t % S) * C::KV_STAGE);
+                const uint32_t d = tmem_base + (uint32_t)((t & 1) ? C::S1_COL : 0);
                 tc_fence_after();
                 int step = 0;
 #pragma unroll
                 for (int a = 0; a < C::NA; a++)
 #pragma unroll
                     for (int k = 0; k < 4; k++, step++)
-                        umma_bf16(tmem_base, umma_desc_k128(q0 + a * C::QA_BYTES) + (uint64_t)(k * 2),
+                        umma_bf16(d, umma_desc_k128(q0 + a * C::QA_BYTES) + (uint64_t)(k * 2),
                                   umma_desc_k128(k0 + a * T::A_BYTES) + (uint64_t)(k * 2), idesc_s, step ? 1u : 0u);
                 if (C::NB) {
 #pragma unroll
                     for (int k = 0; k < 2; k++, step++)
-                        umma_bf16(tmem_base, umma_desc_k64(q0 + C::NA * C::QA_BYTES) + (uint64_t)(k * 2),
+                        umma_bf16(d, umma_desc_k64(q0 + C::NA * C::QA_BYTES) + (uint64_t)(k * 2),
                                   umma_desc_k64(k0 + T::NA * T::A_BYTES) + (uint64_t)(k * 2), idesc_s, step ? 1u : 0u);
                 }
-                umma_commit(s_full);
+                umma_commit(&k_empty[t % S]);            // the K tile has been read
+                umma_commit(&s_full[t & 1]);
             };
-            if (ok) ok = mbar_wait(&kv_full[0], 0);
-            if (ok) issue_qk(0);
+            for (int t = 0; t < 2 && t < nt && ok; t++) {
+                ok = mbar_wait(&k_full[t % S], (t / S) & 1);
+                if (ok) issue_qk(t);
+            }
             for (int t = 0; t < nt && ok; t++) {
                 const int s = t % S;
-                if (*abort_flag || !mbar_wait(p_full, t & 1)) { ok = false; break; }          // P(t) in shared memory, S free
+                if (*abort_flag || !mbar_wait(p_full, t & 1)) { ok = false; break; }          // P(t) in shared memory, S(t) read
+                if (!mbar_wait(&v_full[s], (t / S) & 1)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t v0 = smem_u32(ring + s * C::KV_STAGE + T::BYTES);
 #pragma unroll
@@ -208,11 +243,11 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
                         umma_bf16(tmem_base + (uint32_t)(C::O_COL + T::NA * 64), umma_desc_k128(p0) + (uint64_t)(k * 2),
                                   umma_desc_mn64(v0 + T::NA * T::A_BYTES + k * 1024), idesc_o32, (t | k) ? 1u : 0u);
                 }
-                umma_commit(&kv_empty[s]);               // K and V of this stage have been read
-                if (t + 1 < nt) {
-                    if (*abort_flag || !mbar_wait(&kv_full[(t + 1) % S], ((t + 1) / S) & 1)) { ok = false; break; }
-                    issue_qk(t + 1);                     // its commit also covers the P V just issued
-                } else {
+                umma_commit(&v_empty[s]);                // V of this stage and P have been read, O holds tile t
+                if (t + 2 < nt) {
+                    if (*abort_flag || !mbar_wait(&k_full[(t + 2) % S], ((t + 2) / S) & 1)) { ok = false; break; }
+                    issue_qk(t + 2);
+                } else if (t + 1 == nt) {
                     umma_commit(o_full);                 // the last P V: O is complete
                 }
             }
@@ -224,25 +259,34 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
         const int row = quad * 32 + lane;                 // row of the group = TMEM lane
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
         float m = -INFINITY, l = 0.f;                  // m: the maximum the row's P and O are scaled by (log2 domain)
+        const int wmin_pos = __reduce_min_sync(0xffffffffu, my_pos);
         bool ok = true;
         for (int t = 0; t < nt && ok; t++) {
-            if (*abort_flag || !mbar_wait(s_full, t & 1)) { ok = false; break; }
+            if (*abort_flag || !mbar_wait(&s_full[t & 1], (t >> 1) & 1)) { ok = false; break; }
             tc_fence_after();
             uint32_t sr[64];
-            tmem_ld32(t_lane, sr);
-            tmem_ld32(t_lane + 32, sr + 32);
+            const uint32_t t_s = t_lane + (uint32_t)((t & 1) ? C::S1_COL : 0);
+            tmem_ld32(t_s, sr);
+            tmem_ld32(t_s + 32, sr + 32);
             const int key0 = t * ATT_KT;
+            // causal mask: only tiles that reach past the smallest position of the warp's rows need it
+            if (key0 + ATT_KT - 1 > wmin_pos) {
+#pragma unroll
+                for (int j = 0; j < 64; j++)
+                    if (key0 + j > my_pos) sr[j] = 0xff800000u;      // -inf
+            }
             float mx = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 64; j++) {
-                const float v = (key0 + j <= my_pos) ? __uint_as_float(sr[j]) * scale_log2 : -INFINITY;
-                sr[j] = __float_as_uint(v);
-                mx = fmaxf(mx, v);
-            }
+            for (int j = 0; j < 64; j++) mx = fmaxf(mx, __uint_as_float(sr[j]));
+            mx *= scale_log2;                                        // scale > 0: the maximum commutes with it
+            // S(t) was computed while the previous tile's softmax ran; its P V may still be in flight: O and
+            // the P buffer are at rest once the commit behind that P V has arrived
+            if (t > 0 && !mbar_wait(&v_empty[(t - 1) % S], ((t - 1) / S) & 1)) { ok = false; break; }
+            tc_fence_after();
             // move the row's maximum only when the tile exceeds it by more than 8 (a factor 256)
             const bool move = mx > m + 8.0f || (m == -INFINITY && mx > -INFINITY);
             if (__any_sync(0xffffffffu, move && t > 0 && l > 0.f)) {
-                // rescale O in place: every MMA before this tile's S has completed, so O is at rest
+                // rescale O in place (at rest: see the wait above)
                 const float corr = move ? exp2f(m - mx) : 1.0f;       // (m = -inf: the row has nothing yet, corr 0 is harmless)
 #pragma unroll
                 for (int c = 0; c < D; c += 32) {
@@ -266,7 +310,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
                 uint32_t w[4];
 #pragma unroll
                 for (int q = 0; q < 4; q++) {
-                    const float p0 = exp2f(__uint_as_float(sr[c * 8 + 2 * q]) - u), p1 = exp2f(__uint_as_float(sr[c * 8 + 2 * q + 1]) - u);
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c * 8 + 2 * q]), scale_log2, -u)),
+                                p1 = ex2_approx(fmaf(__uint_as_float(sr[c * 8 + 2 * q + 1]), scale_log2, -u));
                     sum += p0 + p1;
                     w[q] = pack_bf16(p0, p1);
                 }
@@ -275,7 +320,8 @@ attn_prefill_tc_kernel(const __grid_constant__ AtcMaps maps, const int* __restri
             l += sum;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // P visible to the tensor core's reads
             tc_fence_before();
-            mbar_arrive(p_full);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);                               // one arrival per softmax warp
         }
         float o[D];
         if (ok && nt > 0 && !mbar_wait(o_full, 0)) ok = false;
