@@ -163,6 +163,36 @@ def test_sliced_prefill_equals_whole_prefill_bit_for_bit():
     gm.close()
 
 
+def test_sliced_prefill_under_ar_steps():
+    """rd_ar_step works the jobs off as rd_df_step does: a sequence admitted in slices while another
+    decodes sequentially produces the tokens it produces alone, and does not change the other's."""
+    model, w = make_oracle(SMALL, seed=6, max_ctx=128, std=0.08)
+    gm = gpu_model(SMALL, w)
+    pa = rd_inputs.make_prompt(20, SMALL["vocab"], seed=1)
+    pb = rd_inputs.make_prompt(33, SMALL["vocab"], seed=2)
+
+    def run(admit_b, alone_b=False):
+        sess = rd.Session(gm, batch=2, max_context=128, max_window=4, max_new_tokens=10, seed=8)
+        if not alone_b:
+            sess.prefill(0, pa, 3)
+        for step in range(30):
+            if step == 2 and admit_b:
+                (sess.prefill if alone_b else sess.prefill_sliced)(1, pb, 3)
+            if alone_b and step < 2:
+                continue                                   # nothing prefilled yet: a step would be out of order
+            sess.ar_step(3)
+        out = sess.tokens(0).copy(), sess.tokens(1).copy(), sess.committed(1)
+        sess.close()
+        return out
+
+    a_alone, _, _ = run(False)
+    a_both, b_both, (nb, done_b) = run(True)
+    _, b_alone, _ = run(True, alone_b=True)
+    assert np.array_equal(a_alone, a_both) and len(a_both) == 20 + 10
+    assert done_b and nb == 33 + 10 and np.array_equal(b_both, b_alone)
+    gm.close()
+
+
 def test_fp32_pool_adaptive_exit_sampling():
     ls = _run_staggered(SMALL, False, Tolerance(1e-4), 0.0, W=4, n_slots=7, eps=0.05, temperature=0.8, max_new=9, wkw=dict(std=0.08))
     assert ls.near_ties == 0
