@@ -163,6 +163,24 @@ def test_sliced_prefill_equals_whole_prefill_bit_for_bit():
     gm.close()
 
 
+def test_sliced_prefill_of_a_one_token_prompt():
+    """A one-token prompt has no rows to prefill: the job finishes, without a unit, at the next step."""
+    model, w = make_oracle(SMALL, seed=5, max_ctx=64, std=0.08)
+    gm = gpu_model(SMALL, w)
+    out = []
+    for sliced in (False, True):
+        sess = rd.Session(gm, batch=1, max_context=64, max_window=4, max_new_tokens=8, seed=4)
+        (sess.prefill_sliced if sliced else sess.prefill)(0, np.array([7], dtype=np.int32), 2)
+        assert sess.prefill_pending() == (1 if sliced else 0)
+        for _ in range(14):
+            sess.df_step(4, 1, 0.0)
+        assert sess.prefill_pending() == 0 and sess.committed(0) == (9, True)
+        out.append(sess.tokens(0).copy())
+        sess.close()
+    assert np.array_equal(out[0], out[1])
+    gm.close()
+
+
 def test_sliced_prefill_under_ar_steps():
     """rd_ar_step works the jobs off as rd_df_step does: a sequence admitted in slices while another
     decodes sequentially produces the tokens it produces alone, and does not change the other's."""
